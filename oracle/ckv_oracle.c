@@ -1,0 +1,487 @@
+/*
+ * ckv_oracle.c -- TEST INFRASTRUCTURE, not the product.
+ *
+ * A plain, slow, fp64 CPU statement of the end-of-prefill KV retention pass of
+ * CompilerKV (arxiv 2602.08686).  It exists so that the CUDA library can be
+ * checked against something written directly from the paper.  It shares no code
+ * with the CUDA path, and only the tests, the smoke check and the benchmark's
+ * cpu-baseline leg may call it.
+ *
+ * Notation (the build's, not the paper's):  L = prompt length (paper: T),
+ * W = observation-window size |Omega|, n = L - W = prefix length, H = query
+ * heads, Hkv = KV heads, G = H / Hkv, d = head_dim, B = kept rows per KV head on
+ * average (window included).  A "unit" is one (sequence, layer) pair.
+ *
+ * Steps, in the paper's order:
+ *   O1  logits     s[h,i,t] = q[h,i].k[g,t] / sqrt(d), g = h / G        (Sec. 3)
+ *   O2  softmax    over the keys a window row can see (causal)          (Sec. 3)
+ *   O3  column sum c_h[t] = sum_{i in Omega} A[h,i,t]           (Eq. 4, Alg. 1 (A))
+ *   O4  scale      alpha_h[t] = (L / W) c_h[t]                          (Eq. 4)
+ *   O5  1-D pooling of alpha_h over the prefix (argument; size 1 = the paper)
+ *   O6  head table u_g[t] = max_{h in group g} W_head[h] * pooled_h[t]  (Eq. 6)
+ *   O7  risk coordinate: entropy of the normalised window mass, bucket,
+ *       threshold tau = table[bucket]                    (Eq. 7 left, Alg. 1 (A),(D))
+ *   O8  candidate counts under tau (Eq. 8's candidate set) -> per-head budgets
+ *       clamped so that they sum to the total budget
+ *   O9  Top-k per KV head, ties to the lowest index, window always kept (Eq. 8)
+ *   O10 gather of the kept K/V rows                               (Sec. 3, Alg. 1 (D))
+ *
+ * Pins (tests/test_oracle_*.py): the mass identity sum_t c_h[t] = W (text after
+ * Eq. 4), closed-form attention on constant / single-spike inputs, torch's fp64
+ * softmax and pooling routines on special cases, Shannon entropy of uniform and
+ * one-hot distributions, brute-force rational water-filling for O8, brute-force
+ * sorting for O9, direct indexing for O10, FullKV reproduction, and the
+ * identity |p - p~|_1 = 2m of Eq. A2.
+ * Parity unpinned by the paper itself (the paper has no such step; pinned only
+ * by the invariants above): the O8 redistribution rule, the bucket edges of O7,
+ * and the edge rule of the O5 pooling.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define OR_BF16 0
+#define OR_F32 1
+#define OR_POOL_NONE 0
+#define OR_POOL_MAX 1
+#define OR_POOL_AVG 2
+
+typedef struct {
+  int32_t n_units, n_q_heads, n_kv_heads, head_dim, seq_len, window;
+  int32_t dtype; /* OR_BF16: uint16 bit patterns; OR_F32: float */
+} or_shape;
+
+typedef struct {
+  int32_t pool_kind, pool_size;
+  int32_t budget_per_head; /* B */
+  int32_t floor_per_head;  /* f: minimum prefix rows per KV head */
+  int32_t n_buckets;
+  int32_t bucket_override; /* -1: bucket from the entropy */
+  int32_t head_w_per_unit; /* 0: one [H] row shared by all units; 1: [Nu,H] */
+  int32_t sens_per_unit;   /* 0: one [n_buckets] row; 1: [Nu,n_buckets] */
+} or_params;
+
+/* exact widening of an input element to double */
+static double widen(const void *base, int dtype, int64_t idx) {
+  if (dtype == OR_F32) return (double)((const float *)base)[idx];
+  uint32_t bits = ((uint32_t)((const uint16_t *)base)[idx]) << 16;
+  float f;
+  memcpy(&f, &bits, 4);
+  return (double)f;
+}
+
+/* ------------------------------------------------------------------ O1 + O2
+ * One window row of the causal attention matrix: row i of the window sits at
+ * absolute position n + i and sees keys t <= n + i.  A[t] = 0 for hidden keys. */
+static void attention_row(const or_shape *s, const void *q, const void *k, int u, int h, int i,
+                          double *A /* [L] */) {
+  const int L = s->seq_len, W = s->window, d = s->head_dim, H = s->n_q_heads, Hkv = s->n_kv_heads;
+  const int G = H / Hkv, g = h / G, n = L - W;
+  const int last = n + i; /* last visible key */
+  const int64_t qoff = (((int64_t)u * H + h) * W + i) * d;
+  const int64_t koff = ((int64_t)u * Hkv + g) * (int64_t)L * d;
+  const double inv_sqrt_d = 1.0 / sqrt((double)d);
+  double m = -INFINITY;
+  for (int t = 0; t <= last; ++t) {
+    double acc = 0.0;
+    for (int c = 0; c < d; ++c) acc += widen(q, s->dtype, qoff + c) * widen(k, s->dtype, koff + (int64_t)t * d + c);
+    A[t] = acc * inv_sqrt_d;
+    if (A[t] > m) m = A[t];
+  }
+  double l = 0.0;
+  for (int t = 0; t <= last; ++t) {
+    A[t] = exp(A[t] - m);
+    l += A[t];
+  }
+  for (int t = 0; t <= last; ++t) A[t] /= l;
+  for (int t = last + 1; t < L; ++t) A[t] = 0.0;
+}
+
+/* The W x L block of attention rows of every (unit, head): A [Nu,H,W,L]. */
+int oracle_window_attention(const or_shape *s, const void *q, const void *k, double *A) {
+  const int L = s->seq_len, W = s->window, H = s->n_q_heads;
+  if (s->n_q_heads % s->n_kv_heads || W > L || W < 1) return 1;
+#pragma omp parallel for collapse(2) schedule(dynamic)
+  for (int u = 0; u < s->n_units; ++u)
+    for (int h = 0; h < H; ++h)
+      for (int i = 0; i < W; ++i) attention_row(s, q, k, u, h, i, A + ((((int64_t)u * H + h) * W + i) * (int64_t)L));
+  return 0;
+}
+
+/* ------------------------------------------------------------------ O3
+ * c_h[t] = sum over the window rows of A[h,i,t]; csum [Nu,H,L]. */
+int oracle_colsum(const or_shape *s, const void *q, const void *k, double *csum) {
+  const int L = s->seq_len, W = s->window, H = s->n_q_heads;
+  if (s->n_q_heads % s->n_kv_heads || W > L || W < 1) return 1;
+  int err = 0;
+#pragma omp parallel for collapse(2) schedule(dynamic)
+  for (int u = 0; u < s->n_units; ++u)
+    for (int h = 0; h < H; ++h) {
+      double *row = (double *)malloc(sizeof(double) * (size_t)L);
+      double *c = csum + ((int64_t)u * H + h) * (int64_t)L;
+      if (!row) {
+        err = 2;
+        continue;
+      }
+      for (int t = 0; t < L; ++t) c[t] = 0.0;
+      for (int i = 0; i < W; ++i) {
+        attention_row(s, q, k, u, h, i, row);
+        for (int t = 0; t < L; ++t) c[t] += row[t];
+      }
+      free(row);
+    }
+  return err;
+}
+
+/* ------------------------------------------------------------------ O5
+ * Centred stride-1 pooling of x[0..n) with an odd kernel: MAX ignores
+ * positions outside the array (padding with -inf); AVG treats them as zeros
+ * and always divides by the kernel size.  Size 1 / NONE is the identity. */
+int oracle_pool1d(int kind, int size, int n, const double *x, double *out) {
+  if (kind == OR_POOL_NONE || size == 1) {
+    for (int t = 0; t < n; ++t) out[t] = x[t];
+    return 0;
+  }
+  if (size < 1 || (size & 1) == 0) return 1;
+  const int r = size / 2;
+  for (int t = 0; t < n; ++t) {
+    if (kind == OR_POOL_MAX) {
+      double m = -INFINITY;
+      for (int j = t - r; j <= t + r; ++j)
+        if (j >= 0 && j < n && x[j] > m) m = x[j];
+      out[t] = m;
+    } else if (kind == OR_POOL_AVG) {
+      double a = 0.0;
+      for (int j = t - r; j <= t + r; ++j)
+        if (j >= 0 && j < n) a += x[j];
+      out[t] = a / (double)size;
+    } else
+      return 1;
+  }
+  return 0;
+}
+
+/* ------------------------------------------------------------------ O4-O6 (+ the mass for O7)
+ * scores  [Nu,Hkv,n] : u_g[t] = max_{h in g} head_w[h] * pool((L/W) c_h)[t]
+ * colmass [Nu,L]     : sum_h c_h[t]   (all heads of the unit, window columns included)
+ * csum    [Nu,H,L]   : c_h[t] (optional) */
+int oracle_score(const or_shape *s, const or_params *p, const void *q, const void *k, const float *head_w,
+                 double *scores, double *colmass, double *csum_or_null) {
+  const int L = s->seq_len, W = s->window, H = s->n_q_heads, Hkv = s->n_kv_heads, Nu = s->n_units;
+  if (H % Hkv || W > L || W < 1) return 1;
+  const int G = H / Hkv, n = L - W;
+  double *csum = csum_or_null ? csum_or_null : (double *)malloc(sizeof(double) * (size_t)Nu * H * L);
+  if (!csum) return 2;
+  int rc = oracle_colsum(s, q, k, csum);
+  if (rc) goto done;
+#pragma omp parallel for schedule(dynamic)
+  for (int u = 0; u < Nu; ++u) {
+    double *alpha = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
+    double *pooled = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
+    for (int t = 0; t < L; ++t) {
+      double m = 0.0;
+      for (int h = 0; h < H; ++h) m += csum[((int64_t)u * H + h) * L + t];
+      colmass[(int64_t)u * L + t] = m;
+    }
+    for (int g = 0; g < Hkv; ++g) {
+      double *out = scores + ((int64_t)u * Hkv + g) * (int64_t)n;
+      for (int t = 0; t < n; ++t) out[t] = -INFINITY;
+      for (int h = g * G; h < (g + 1) * G; ++h) {
+        const double w = (double)head_w[p->head_w_per_unit ? (int64_t)u * H + h : h];
+        const double *c = csum + ((int64_t)u * H + h) * (int64_t)L;
+        for (int t = 0; t < n; ++t) alpha[t] = ((double)L / (double)W) * c[t];
+        oracle_pool1d(p->pool_kind, p->pool_size, n, alpha, pooled);
+        for (int t = 0; t < n; ++t) {
+          const double v = w * pooled[t];
+          if (v > out[t]) out[t] = v;
+        }
+      }
+    }
+    free(alpha);
+    free(pooled);
+  }
+done:
+  if (!csum_or_null) free(csum);
+  return rc;
+}
+
+/* ------------------------------------------------------------------ O7
+ * p[t] = colmass[t] / (W H) is a distribution over the L keys (each of the W H
+ * softmax rows sums to one).  ent = -sum p ln p, hn = ent / ln L in [0,1],
+ * bucket = min(nb - 1, floor(hn nb)). */
+static void risk_bucket(const double *colmass, int L, int W, int H, int nb, double *ent_out, int *bucket_out) {
+  double ent = 0.0;
+  for (int t = 0; t < L; ++t) {
+    const double pt = colmass[t] / ((double)W * (double)H);
+    if (pt > 0.0) ent -= pt * log(pt);
+  }
+  double hn = (L > 1) ? ent / log((double)L) : 0.0;
+  int b = (int)floor(hn * (double)nb);
+  if (b > nb - 1) b = nb - 1;
+  if (b < 0) b = 0;
+  *ent_out = ent;
+  *bucket_out = b;
+}
+
+/* ------------------------------------------------------------------ O8
+ * Split P prefix rows over Hkv heads in proportion to demands dem[g] >= 1,
+ * every share held inside [f, n]:  x_g = clamp(lambda dem_g, f, n) with lambda
+ * the water level at which the shares sum to P (unique shares because the sum
+ * is continuous and non-decreasing in lambda).  All comparisons are between
+ * integers.  The real shares of the unclamped heads are then rounded down and
+ * the left-over rows go, one each, to the largest fractional parts, ties to the
+ * lowest head index.  Requires f Hkv <= P <= n Hkv.  Returns 0 on success. */
+int oracle_allocate(int Hkv, int64_t n, int64_t f, int64_t P, const int64_t *dem, int64_t *e) {
+  if (Hkv < 1 || f < 0 || f > n || P < f * Hkv || P > n * Hkv) return 1;
+  for (int g = 0; g < Hkv; ++g)
+    if (dem[g] < 1) return 1;
+  /* lambda = num/den runs over the break points f/dem_g and n/dem_g; at each
+   * candidate level classify every head and test whether the level that makes
+   * the unclamped heads absorb the rest lies in the same linear piece. */
+  for (int cand = 0; cand < 2 * Hkv + 1; ++cand) {
+    /* the piece just above break point `cand` (cand == 2 Hkv: the piece below all of them) */
+    int64_t bn, bd; /* break point = bn / bd */
+    if (cand == 2 * Hkv) {
+      bn = 0;
+      bd = 1;
+    } else {
+      bn = (cand < Hkv) ? f : n;
+      bd = dem[cand % Hkv];
+    }
+    /* classify at a level infinitesimally above bn/bd:
+       low  (share f): lambda dem_g <= f  <=> bn dem_g <  f bd   (strict: at equality the head is leaving the clamp)
+       high (share n): lambda dem_g >= n  <=> bn dem_g >= n bd
+       else free. */
+    int64_t R = P, D = 0;
+    int state[64];
+    if (Hkv > 64) return 1;
+    for (int g = 0; g < Hkv; ++g) {
+      if (bn * dem[g] >= n * bd) {
+        state[g] = 2;
+        R -= n;
+      } else if (bn * dem[g] < f * bd) {
+        state[g] = 0;
+        R -= f;
+      } else {
+        state[g] = 1;
+        D += dem[g];
+      }
+    }
+    int ok = 1;
+    if (D == 0) {
+      ok = (R == 0);
+    } else {
+      /* lambda* = R / D must keep every free head inside [f, n], every low head
+         at or below f and every high head at or above n */
+      if (R < 0) ok = 0;
+      for (int g = 0; g < Hkv && ok; ++g) {
+        const int64_t lhs = R * dem[g];
+        if (state[g] == 1 && (lhs < f * D || lhs > n * D)) ok = 0;
+        if (state[g] == 0 && lhs > f * D) ok = 0;
+        if (state[g] == 2 && lhs < n * D) ok = 0;
+      }
+    }
+    if (!ok) continue;
+    int64_t given = 0;
+    int64_t rem[64];
+    for (int g = 0; g < Hkv; ++g) {
+      if (state[g] == 0) {
+        e[g] = f;
+        rem[g] = -1;
+      } else if (state[g] == 2) {
+        e[g] = n;
+        rem[g] = -1;
+      } else {
+        e[g] = (R * dem[g]) / D;
+        rem[g] = (R * dem[g]) % D;
+        given += e[g];
+      }
+    }
+    int64_t left = (D > 0) ? R - given : 0;
+    while (left > 0) {
+      int best = -1;
+      for (int g = 0; g < Hkv; ++g)
+        if (rem[g] > 0 && (best < 0 || rem[g] > rem[best])) best = g;
+      if (best < 0) return 3; /* cannot happen: left < number of non-zero remainders */
+      e[best] += 1;
+      rem[best] = -1;
+      --left;
+    }
+    return 0;
+  }
+  return 2;
+}
+
+/* budgets [Nu,Hkv], offsets [Nu,Hkv+1], bucket [Nu], entropy [Nu], tau [Nu], counts [Nu,Hkv] (optional) */
+int oracle_budget(const or_shape *s, const or_params *p, const double *scores, const double *colmass,
+                  const float *sens, int32_t *budgets, int32_t *offsets, int32_t *bucket, double *entropy,
+                  double *tau_out, int32_t *counts_or_null) {
+  const int L = s->seq_len, W = s->window, H = s->n_q_heads, Hkv = s->n_kv_heads, Nu = s->n_units;
+  const int n = L - W, B = p->budget_per_head, f = p->floor_per_head;
+  if (p->n_buckets < 1 || Hkv > 64) return 1;
+  if (B < L && (B < W || f > B - W || f < 0)) return 1;
+  for (int u = 0; u < Nu; ++u) {
+    double ent;
+    int b;
+    risk_bucket(colmass + (int64_t)u * L, L, W, H, p->n_buckets, &ent, &b);
+    if (p->bucket_override >= 0) b = p->bucket_override < p->n_buckets ? p->bucket_override : p->n_buckets - 1;
+    const double tau = (double)sens[(p->sens_per_unit ? (int64_t)u * p->n_buckets : 0) + b];
+    bucket[u] = b;
+    entropy[u] = ent;
+    if (tau_out) tau_out[u] = tau;
+    int64_t dem[64], e[64];
+    for (int g = 0; g < Hkv; ++g) {
+      const double *sc = scores + ((int64_t)u * Hkv + g) * (int64_t)n;
+      int64_t c = 0;
+      for (int t = 0; t < n; ++t) c += (sc[t] >= tau);
+      if (counts_or_null) counts_or_null[(int64_t)u * Hkv + g] = (int32_t)c;
+      int64_t lo = f > 1 ? f : 1;
+      dem[g] = c < lo ? lo : (c > n ? n : c);
+    }
+    if (B >= L) {
+      for (int g = 0; g < Hkv; ++g) e[g] = n; /* FullKV: the whole prefix, then the window */
+    } else {
+      int rc = oracle_allocate(Hkv, n, f, (int64_t)Hkv * (B - W), dem, e);
+      if (rc) return 10 + rc;
+    }
+    int32_t off = 0;
+    for (int g = 0; g < Hkv; ++g) {
+      budgets[(int64_t)u * Hkv + g] = (int32_t)(e[g] + W);
+      offsets[(int64_t)u * (Hkv + 1) + g] = off;
+      off += (int32_t)(e[g] + W);
+    }
+    offsets[(int64_t)u * (Hkv + 1) + Hkv] = off;
+  }
+  return 0;
+}
+
+/* ------------------------------------------------------------------ O9 */
+typedef struct {
+  double score;
+  int32_t idx;
+} or_item;
+
+static int by_score_desc_then_index(const void *a, const void *b) {
+  const or_item *x = (const or_item *)a, *y = (const or_item *)b;
+  if (x->score > y->score) return -1;
+  if (x->score < y->score) return 1;
+  return (x->idx > y->idx) - (x->idx < y->idx);
+}
+static int by_index(const void *a, const void *b) {
+  const or_item *x = (const or_item *)a, *y = (const or_item *)b;
+  return (x->idx > y->idx) - (x->idx < y->idx);
+}
+
+/* indices [Nu, sum_g budgets] packed at offsets: per KV head the budgets[g] - W
+ * best prefix positions in ascending order, then n .. L-1. */
+int oracle_select(const or_shape *s, const double *scores, const int32_t *budgets, const int32_t *offsets,
+                  int32_t *indices) {
+  const int L = s->seq_len, W = s->window, Hkv = s->n_kv_heads, Nu = s->n_units, n = L - W;
+  int err = 0;
+#pragma omp parallel for collapse(2) schedule(dynamic)
+  for (int u = 0; u < Nu; ++u)
+    for (int g = 0; g < Hkv; ++g) {
+      const int e = budgets[(int64_t)u * Hkv + g] - W;
+      const int64_t rows_per_unit = offsets[(int64_t)u * (Hkv + 1) + Hkv];
+      int32_t *out = indices + (int64_t)u * rows_per_unit + offsets[(int64_t)u * (Hkv + 1) + g];
+      if (e < 0 || e > n) {
+        err = 1;
+        continue;
+      }
+      or_item *it = (or_item *)malloc(sizeof(or_item) * (size_t)(n > 0 ? n : 1));
+      const double *sc = scores + ((int64_t)u * Hkv + g) * (int64_t)n;
+      for (int t = 0; t < n; ++t) {
+        it[t].score = sc[t];
+        it[t].idx = t;
+      }
+      qsort(it, (size_t)n, sizeof(or_item), by_score_desc_then_index);
+      qsort(it, (size_t)e, sizeof(or_item), by_index);
+      for (int j = 0; j < e; ++j) out[j] = it[j].idx;
+      for (int i = 0; i < W; ++i) out[e + i] = n + i;
+      free(it);
+    }
+  return err;
+}
+
+/* ------------------------------------------------------------------ O10 */
+int oracle_gather(const or_shape *s, const void *k, const void *v, const int32_t *indices, const int32_t *budgets,
+                  const int32_t *offsets, void *k_out, void *v_out) {
+  const int L = s->seq_len, d = s->head_dim, Hkv = s->n_kv_heads, Nu = s->n_units;
+  const size_t esz = s->dtype == OR_F32 ? 4 : 2, row = esz * (size_t)d;
+  for (int u = 0; u < Nu; ++u) {
+    const int64_t rows_per_unit = offsets[(int64_t)u * (Hkv + 1) + Hkv];
+    for (int g = 0; g < Hkv; ++g) {
+      const int64_t o = (int64_t)u * rows_per_unit + offsets[(int64_t)u * (Hkv + 1) + g];
+      for (int j = 0; j < budgets[(int64_t)u * Hkv + g]; ++j) {
+        const int32_t t = indices[o + j];
+        if (t < 0 || t >= L) return 1;
+        const size_t src = (((size_t)u * Hkv + g) * (size_t)L + (size_t)t) * row;
+        memcpy((char *)k_out + (size_t)(o + j) * row, (const char *)k + src, row);
+        memcpy((char *)v_out + (size_t)(o + j) * row, (const char *)v + src, row);
+      }
+    }
+  }
+  return 0;
+}
+
+/* ------------------------------------------------------------------ whole pass
+ * Outputs are sized for B' = min(B, L) rows per KV head:
+ * k_out, v_out [Nu, Hkv B', d]; indices [Nu, Hkv B']; budgets [Nu,Hkv];
+ * offsets [Nu,Hkv+1]; scores [Nu,Hkv,n] (fp64, optional). */
+int oracle_compress(const or_shape *s, const or_params *p, const void *q, const void *k, const void *v,
+                    const float *head_w, const float *sens, void *k_out, void *v_out, int32_t *indices,
+                    int32_t *budgets, int32_t *offsets, int32_t *bucket, double *entropy, double *scores_or_null) {
+  const int L = s->seq_len, W = s->window, Hkv = s->n_kv_heads, Nu = s->n_units, n = L - W;
+  double *scores = scores_or_null ? scores_or_null : (double *)malloc(sizeof(double) * (size_t)Nu * Hkv * (n > 0 ? n : 1));
+  double *colmass = (double *)malloc(sizeof(double) * (size_t)Nu * L);
+  int rc = 2;
+  if (scores && colmass) {
+    rc = oracle_score(s, p, q, k, head_w, scores, colmass, NULL);
+    if (!rc) rc = oracle_budget(s, p, scores, colmass, sens, budgets, offsets, bucket, entropy, NULL, NULL);
+    if (!rc) rc = oracle_select(s, scores, budgets, offsets, indices);
+    if (!rc) rc = oracle_gather(s, k, v, indices, budgets, offsets, k_out, v_out);
+  }
+  if (!scores_or_null) free(scores);
+  free(colmass);
+  return rc;
+}
+
+/* ------------------------------------------------------------------ diagnostic (Prop. 4.1)
+ * kept[u,h,i] = sum_{t in S_g} A[h,i,t]: attention mass of window row i that
+ * survives the selection; the discarded mass is m = 1 - kept. */
+int oracle_kept_mass(const or_shape *s, const void *q, const void *k, const int32_t *indices, const int32_t *budgets,
+                     const int32_t *offsets, double *kept) {
+  const int L = s->seq_len, W = s->window, H = s->n_q_heads, Hkv = s->n_kv_heads, G = H / Hkv;
+#pragma omp parallel for collapse(2) schedule(dynamic)
+  for (int u = 0; u < s->n_units; ++u)
+    for (int h = 0; h < H; ++h) {
+      const int g = h / G;
+      double *row = (double *)malloc(sizeof(double) * (size_t)L);
+      const int64_t rows_per_unit = offsets[(int64_t)u * (Hkv + 1) + Hkv];
+      const int32_t *idx = indices + (int64_t)u * rows_per_unit + offsets[(int64_t)u * (Hkv + 1) + g];
+      for (int i = 0; i < W; ++i) {
+        attention_row(s, q, k, u, h, i, row);
+        double a = 0.0;
+        for (int j = 0; j < budgets[(int64_t)u * Hkv + g]; ++j) a += row[idx[j]];
+        kept[((int64_t)u * H + h) * W + i] = a;
+      }
+      free(row);
+    }
+  return 0;
+}
+
+int oracle_num_threads(void) {
+  int nt = 1;
+#ifdef _OPENMP
+#pragma omp parallel
+  {
+#pragma omp single
+    nt = omp_get_num_threads();
+  }
+#endif
+  return nt;
+}
