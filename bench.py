@@ -1,0 +1,319 @@
+#!/usr/bin/env python
+"""Benchmark of the end-of-prefill KV retention pass (one JSON line on stdout).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload c2|c4|...]
+
+A step is one call of the fused ``ckv_compress`` over one batch of synthetic units (sequence x layer
+pairs) resident in HBM.  The default workload is the Llama-3-8B-shaped pass at L = 32768 (32 units,
+512 rows kept per KV head).  Under torchrun every rank runs the same number of its own units (weak
+scaling, no data-path collective); the time is the max over ranks.  ``--impl reference`` times the
+fp64 CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2602_08686_b200 import inputs as gen  # noqa: E402
+from paper_2602_08686_b200.sharding import max_over_ranks  # noqa: E402
+
+METRIC = "prefill_tokens_compressed_per_sec_per_layer"
+UNIT = "tokens/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.rows, self.proc, self.thread = [], None, None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(index)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        rows = [r for t, r in self.rows if t0 <= t <= t1 + 0.1] or [r for _, r in self.rows[-3:]]
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            c = [x.strip() for x in r.split(",")]
+            try:
+                sm.append(float(c[0]))
+                smax.append(float(c[1]))
+            except (ValueError, IndexError):
+                continue
+            for nme, val in zip(names, c[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nme)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_problem(cfg, Nu):
+    import oracle
+    return oracle.Problem(Nu, cfg.n_q_heads, cfg.n_kv_heads, cfg.seq_len, cfg.window, head_dim=cfg.head_dim,
+                          dtype=oracle.BF16 if cfg.dtype == "bf16" else oracle.F32, pool_kind=cfg.pool_kind,
+                          pool_size=cfg.pool_size, budget_per_head=cfg.budget_per_head,
+                          floor_per_head=cfg.floor_per_head, n_buckets=cfg.n_buckets)
+
+
+def time_oracle(cfg, batch_cpu, n_sample_units, repeats=1):
+    """Seconds per run of the oracle's whole pass on the first n_sample_units units (host tensors)."""
+    import oracle
+    prob = oracle_problem(cfg, n_sample_units)
+    args = [gen.as_numpy(batch_cpu[x][:n_sample_units]) for x in ("q", "k", "v", "head_w")]
+    args.append(gen.as_numpy(batch_cpu["sens"]))
+    best = float("inf")
+    for _ in range(repeats):
+        t = time.perf_counter()
+        oracle.compress(prob, *args, want_scores=False)
+        best = min(best, time.perf_counter() - t)
+    return best, oracle.num_threads()
+
+
+def algorithmic_bytes(cfg, n_units):
+    """K read twice plus the kept K/V rows read and written (the benchmark's roofline definition)."""
+    esz = 2 if cfg.dtype == "bf16" else 4
+    k_bytes = n_units * cfg.n_kv_heads * cfg.seq_len * cfg.head_dim * esz
+    rows = n_units * cfg.n_kv_heads * min(cfg.budget_per_head, cfg.seq_len)
+    gather = 4 * rows * cfg.head_dim * esz
+    return 2 * k_bytes, gather
+
+
+def config_dict(cfg, n_units_per_gpu, world):
+    return {"workload": cfg.name, "shape": f"{cfg.n_q_heads}q/{cfg.n_kv_heads}kv heads, d {cfg.head_dim}",
+            "seq_len": cfg.seq_len, "window": cfg.window, "budget_per_head": cfg.budget_per_head,
+            "pool": f"{'none max avg'.split()[cfg.pool_kind]}{cfg.pool_size}", "units_per_gpu": n_units_per_gpu,
+            "units_total": n_units_per_gpu * world, "parallelism": f"dp{world} over units (no collective)",
+            "l2": "inputs (K+V %.1f GB per GPU) exceed the 126 MB L2; no flush needed" %
+                  (2 * n_units_per_gpu * cfg.n_kv_heads * cfg.seq_len * cfg.head_dim *
+                   (2 if cfg.dtype == "bf16" else 4) / 1e9)}
+
+
+def run_reference(args, cfg, rank, world):
+    """The oracle, as it stands, on the host cores: each step is one unit of the workload."""
+    if rank != 0:
+        return
+    sample_units = 1
+    units = list(range(sample_units))
+    batch = gen.make_batch(cfg, "cpu", units)
+    for _ in range(max(args.warmup, 0)):
+        time_oracle(cfg, batch, sample_units)
+    t0 = time.perf_counter()
+    cores = 1
+    for _ in range(args.steps):
+        _, cores = time_oracle(cfg, batch, sample_units)
+    el = time.perf_counter() - t0
+    value = args.steps * sample_units * cfg.seq_len / el
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * el / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": config_dict(cfg, sample_units, 1),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": f"{sample_units} unit(s) of {cfg.name} per step (whole pass, fp64)"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2", choices=sorted(gen.CONFIGS))
+    ap.add_argument("--units", type=int, default=0, help="units per GPU (default: the workload's)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    cfg = gen.CONFIGS[args.workload]
+
+    if args.impl == "reference":
+        run_reference(args, cfg, rank, world)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the retention pass has no CPU fallback")
+    from paper_2602_08686_b200 import binding as B
+    B.lib()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    import torch.distributed as dist
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    n_units = args.units or cfg.n_units
+    units = [rank * n_units + u for u in range(n_units)]
+    batch = gen.make_batch(cfg, dev, units)
+    P = B.Params(pool_kind=cfg.pool_kind, pool_size=cfg.pool_size, budget_per_head=cfg.budget_per_head,
+                 floor_per_head=cfg.floor_per_head, n_buckets=cfg.n_buckets)
+    shape = B.make_shape(batch["q"], batch["k"])
+    params = B.make_params(P, batch["head_w"], batch["sens"])
+    ws = B.alloc_workspace(shape, params, dev)
+    Hkv, L, n = cfg.n_kv_heads, cfg.seq_len, cfg.n
+    rows = B.rows_per_unit(shape, params)
+    k_out = torch.empty(n_units, rows, cfg.head_dim, dtype=batch["k"].dtype, device=dev)
+    v_out = torch.empty_like(k_out)
+    indices = torch.empty(n_units, rows, dtype=torch.int32, device=dev)
+    budgets = torch.empty(n_units, Hkv, dtype=torch.int32, device=dev)
+    offsets = torch.empty(n_units, Hkv + 1, dtype=torch.int32, device=dev)
+    scores = torch.empty(n_units, Hkv, n, dtype=torch.float32, device=dev)
+    colmass = torch.empty(n_units, L, dtype=torch.float32, device=dev)
+    bucket = torch.empty(n_units, dtype=torch.int32, device=dev)
+    entropy = torch.empty(n_units, dtype=torch.float32, device=dev)
+
+    def step():
+        B.ckv_compress(shape, params, batch["q"], batch["k"], batch["v"], batch["head_w"], batch["sens"], k_out,
+                       v_out, indices, budgets, offsets, ws)
+
+    # ---- device-resident timing ---------------------------------------------------------------
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    launches0 = B.ckv_kernel_launches()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    t1 = time.time()
+    launches = B.ckv_kernel_launches() - launches0
+    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    clocks = sampler.stop(t0, t1) if sampler else None
+    if B.ckv_device_status(ws) != B.OK:
+        raise SystemExit("device-side wait timed out")
+    ms_per_step = ms_total / args.steps
+    value = world * n_units * L / (ms_per_step * 1e-3)
+
+    # ---- per-stage timing (same kernels through the staged entry points) --------------------------
+    stage_names = ["score", "budget", "select", "gather"]
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+    for it in range(args.steps):
+        ev = evs[it]
+        ev[0].record()
+        B.ckv_score(shape, params, batch["q"], batch["k"], batch["head_w"], scores, colmass, ws)
+        ev[1].record()
+        B.ckv_budget(shape, params, scores, colmass, batch["sens"], budgets, offsets, bucket, entropy, ws)
+        ev[2].record()
+        B.ckv_select(shape, params, scores, budgets, offsets, indices, ws)
+        ev[3].record()
+        B.ckv_gather(shape, params, batch["k"], batch["v"], indices, offsets, k_out, v_out)
+        ev[4].record()
+    torch.cuda.synchronize()
+    stage_ms = {nm: sum(evs[it][j].elapsed_time(evs[it][j + 1]) for it in range(args.steps)) / args.steps
+                for j, nm in enumerate(stage_names)}
+
+    peak, peak_kind = measured_peaks()
+    k2_bytes, gather_bytes = algorithmic_bytes(cfg, n_units)
+    score_gbs = k2_bytes / (stage_ms["score"] * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "ckv_score (window-score scan, both K passes, + pooling epilogue)",
+                "achieved": score_gbs, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                "frac": score_gbs / peak, "traffic": None,
+                "algorithmic_bytes_per_launch": k2_bytes, "ms_per_launch": stage_ms["score"],
+                "whole_pass": {"algorithmic_bytes": k2_bytes + gather_bytes,
+                               "achieved": (k2_bytes + gather_bytes) / (ms_per_step * 1e-3) / 1e9,
+                               "frac": (k2_bytes + gather_bytes) / (ms_per_step * 1e-3) / 1e9 / peak,
+                               "frac_of_nominal_8TBs": (k2_bytes + gather_bytes) / (ms_per_step * 1e-3) / 8e12},
+                "stage_ms": stage_ms}
+
+    # ---- end to end through ckv_compress_host (pinned host buffers, copies inside the timed region) ----
+    e2e = None
+    if not args.no_e2e:
+        pin = lambda t: t.cpu().pin_memory()
+        hq, hk, hv, hw, hs = (pin(batch[x]) for x in ("q", "k", "v", "head_w", "sens"))
+        hko, hvo = pin(k_out), pin(v_out)
+        hidx, hbud, hoff = pin(indices), pin(budgets), pin(offsets)
+        staging = torch.empty(B.ckv_staging_bytes(shape, params), dtype=torch.uint8, device=dev)
+        h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv, hw, hs))
+        d2h = sum(t.numel() * t.element_size() for t in (hko, hvo, hidx, hbud, hoff))
+        e2e_steps = max(1, min(args.steps, 3))
+
+        def host_step():
+            B.ckv_compress_host(shape, params, hq, hk, hv, hw, hs, hko, hvo, hidx, hbud, hoff, staging, ws)
+
+        host_step()
+        barrier()
+        e0.record()
+        for _ in range(e2e_steps):
+            host_step()
+        e1.record()
+        barrier()
+        ms_e2e = max_over_ranks(e0.elapsed_time(e1)) / e2e_steps
+        e2e = {"value": world * n_units * L / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "steps": e2e_steps,
+               "api": "ckv_compress_host (pinned host tensors)"}
+        assert torch.equal(hidx, indices.cpu())
+        del staging
+
+    # ---- the oracle on the host cores, bounded sample (rank 0, single GPU only) ----------------------
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        sample = min(2, n_units)
+        host = {x: batch[x][:sample].cpu() for x in ("q", "k", "v", "head_w")}
+        host["sens"] = batch["sens"].cpu()
+        sec, cores = time_oracle(cfg, host, sample)
+        cpu_baseline = {"value": sample * L / sec, "unit": UNIT, "cores": cores, "kind": "oracle",
+                        "sample": f"first {sample} of {n_units} units of {cfg.name}, whole pass, fp64, "
+                                  f"{sec:.2f} s wall"}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if cfg.dtype == "bf16" else "f32",
+                "data": "synthetic", "config": config_dict(cfg, n_units, world), "clocks": clocks, "e2e": e2e,
+                "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu_baseline}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,173 @@
+/*
+ * ckv.h -- C ABI of libckv: the end-of-prefill KV retention pass of CompilerKV
+ * (arxiv 2602.08686) as hand-written sm_100a CUDA kernels for one B200.
+ *
+ * Notation: L = prompt length (the paper's T), W = observation-window size
+ * |Omega| (the last W prompt positions), n = L - W = prefix length, H = query
+ * heads, Hkv = KV heads, G = H / Hkv (query head h reads KV head h / G),
+ * d = head_dim, B = rows kept per KV head on average (window included).
+ * A "unit" is one (sequence, layer) pair; a call processes Nu independent units.
+ *
+ * General rules for every entry point
+ *   - Every data pointer is a DEVICE pointer unless the argument name ends in
+ *     `_host`.  `shape` and `params` are HOST structs read before the call returns.
+ *   - The caller owns every buffer.  The library allocates no device memory and
+ *     keeps no per-call state; work space is passed in (`ws`, `ws_bytes`, at
+ *     least ckv_workspace_bytes(), 256-byte aligned).
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL is
+ *     the default stream) and return after the last launch was queued.
+ *   - Errors are return codes.  Argument errors are found on the host before
+ *     anything is launched (CKV_ERR_INVALID_ARG / UNSUPPORTED / WORKSPACE); a CUDA
+ *     launch error gives CKV_ERR_CUDA.  A device-side wait that ran out of its
+ *     iteration limit is recorded in the work space's status word and read back
+ *     with ckv_device_status().
+ *   - Preconditions that are not checked: inputs are finite, head_w >= 0.
+ *   - Layouts: q_win [Nu, H, W, d], k and v [Nu, Hkv, L, d]; the last dimension is
+ *     contiguous and the other strides are given in ELEMENTS in ckv_shape; every row
+ *     must start on a 16-byte boundary.  All outputs are dense.
+ */
+#ifndef CKV_H_
+#define CKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  CKV_OK = 0,
+  CKV_ERR_INVALID_ARG = 1, /* null / misaligned pointer, inconsistent shape or parameter */
+  CKV_ERR_UNSUPPORTED = 2, /* valid but not implemented: head_dim != 128, window > 64, Hkv > 64, ... */
+  CKV_ERR_WORKSPACE = 3,   /* ws is null, misaligned or shorter than ckv_workspace_bytes() */
+  CKV_ERR_CUDA = 4,        /* a CUDA runtime call or launch failed */
+  CKV_ERR_TIMEOUT = 5      /* a bounded device-side wait expired (see ckv_device_status) */
+} ckv_status;
+
+typedef enum { CKV_BF16 = 0, CKV_F32 = 1 } ckv_dtype;
+typedef enum { CKV_POOL_NONE = 0, CKV_POOL_MAX = 1, CKV_POOL_AVG = 2 } ckv_pool;
+
+typedef struct {
+  int32_t n_units;    /* Nu >= 1 */
+  int32_t n_q_heads;  /* H, a multiple of n_kv_heads */
+  int32_t n_kv_heads; /* Hkv <= 64 */
+  int32_t head_dim;   /* d; must be 128 */
+  int32_t seq_len;    /* L >= window */
+  int32_t window;     /* W in [1, 64] */
+  int32_t dtype;      /* ckv_dtype of q_win, k, v and of k_out, v_out */
+  int32_t reserved_;  /* set to 0 */
+  int64_t q_stride_unit, q_stride_head, q_stride_row;  /* elements */
+  int64_t kv_stride_unit, kv_stride_head, kv_stride_tok; /* elements; shared by k and v */
+} ckv_shape;
+
+typedef struct {
+  int32_t pool_kind;        /* ckv_pool */
+  int32_t pool_size;        /* odd, 1..15; 1 (or CKV_POOL_NONE) is the paper's un-pooled score */
+  int32_t budget_per_head;  /* B >= 1: rows kept per KV head on average, window included; the unit's
+                               heads share Hkv * min(B, L) rows.  B >= L keeps everything (FullKV). */
+  int32_t floor_per_head;   /* f >= 0: least number of PREFIX rows any KV head keeps; f <= B - W */
+  int32_t n_buckets;        /* size of one row of the threshold table */
+  int32_t bucket_override;  /* -1: bucket from the entropy of the unit's window mass; else that bucket */
+  int64_t head_w_stride_unit; /* elements between the head_w rows of consecutive units; 0 = one row for all */
+  int64_t sens_stride_unit;   /* same for the threshold table */
+} ckv_params;
+
+/* Bytes of work space any entry point needs for this problem (0 on invalid arguments). */
+size_t ckv_workspace_bytes(const ckv_shape* shape, const ckv_params* params);
+
+/*
+ * Window-score scan and head-table weighting (Sec. 3 softmax; Eq. 4's window mass alpha; Eq. 6's
+ * weighted max over heads, taken inside each GQA group; 1-D pooling is an argument the paper does
+ * not have).  For every unit and query head h:
+ *   s[i,t]  = q_win[h,i] . k[h/G,t] / sqrt(d)   for window row i (position n+i) and keys t <= n+i
+ *   A[i,:]  = softmax(s[i,:]);   c_h[t] = sum_i A[i,t];   alpha_h[t] = (L/W) c_h[t]
+ *   P_h     = pool(alpha_h[0:n])  (centred, stride 1; MAX ignores positions outside [0,n), AVG
+ *             counts them as zeros and divides by pool_size)
+ * Outputs: scores [Nu,Hkv,n] fp32, scores[g,t] = max_{h in group g} head_w[h] * P_h[t];
+ *          colmass [Nu,L] fp32, colmass[t] = sum_h c_h[t] over all H heads (window columns included).
+ * head_w: [H] fp32 per unit (params->head_w_stride_unit apart).
+ */
+ckv_status ckv_score(const ckv_shape* shape, const ckv_params* params, const void* q_win, const void* k,
+                     const float* head_w, float* scores, float* colmass, void* ws, size_t ws_bytes,
+                     void* stream);
+
+/*
+ * Risk coordinate, threshold lookup and per-head budgets (Eq. 7's attention entropy; the gate
+ * lookup of Sec. 4.3 / Alg. 1 (D); Eq. 8's candidate set; the clamp to the total budget).
+ *   p[t] = colmass[t] / (W H);  entropy = -sum_t p ln p;  bucket = min(n_buckets-1,
+ *   floor(n_buckets * entropy / ln L)) unless overridden;  tau = sens[bucket];
+ *   count_g = #{t < n : scores[g,t] >= tau};  demand_g = clamp(count_g, max(f,1), n);
+ *   the Hkv (B - W) prefix rows of the unit are split in proportion to the demands with every
+ *   share clamped to [f, n] (water-filling in exact integer arithmetic; shares rounded down, the
+ *   remainder handed out by largest fractional part, ties to the lowest head);
+ *   budgets[g] = W + share_g, so sum_g budgets[g] = Hkv B.  B >= L gives budgets[g] = L.
+ * Outputs: budgets [Nu,Hkv] int32; offsets [Nu,Hkv+1] int32 (exclusive prefix sums of budgets);
+ *          bucket [Nu] int32; entropy [Nu] fp32.  sens: [n_buckets] fp32 per unit.
+ */
+ckv_status ckv_budget(const ckv_shape* shape, const ckv_params* params, const float* scores,
+                      const float* colmass, const float* sens, int32_t* budgets, int32_t* offsets,
+                      int32_t* bucket, float* entropy, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Per-head Top-k (Eq. 8's Top-B branch).  For every unit and KV head g the budgets[g] - W
+ * largest of scores[g,0:n] are kept, equal scores resolved toward the lowest index; the kept
+ * positions are written in ascending order and followed by the window n .. L-1, which is always
+ * retained.  indices [Nu, Hkv * min(B,L)] int32, head g of unit u at row offsets[u,g].
+ */
+ckv_status ckv_select(const ckv_shape* shape, const ckv_params* params, const float* scores,
+                      const int32_t* budgets, const int32_t* offsets, int32_t* indices, void* ws,
+                      size_t ws_bytes, void* stream);
+
+/*
+ * Gather of the retained rows (K~ = K[S], V~ = V[S] of Sec. 3 / Alg. 1 (D)): bit copies.
+ * k_out, v_out [Nu, Hkv * min(B,L), d] in the input dtype, rows in the order of `indices`.
+ */
+ckv_status ckv_gather(const ckv_shape* shape, const ckv_params* params, const void* k, const void* v,
+                      const int32_t* indices, const int32_t* offsets, void* k_out, void* v_out,
+                      void* stream);
+
+/*
+ * The whole pass in one call: score -> budget -> select -> gather on one stream (Alg. 1 (A)-(D)
+ * for the per-unit reading described above).  scores_or_null [Nu,Hkv,n] receives the scores when
+ * given; bucket_or_null [Nu] and entropy_or_null [Nu] likewise.
+ */
+ckv_status ckv_compress(const ckv_shape* shape, const ckv_params* params, const void* q_win, const void* k,
+                        const void* v, const float* head_w, const float* sens, void* k_out, void* v_out,
+                        int32_t* indices, int32_t* budgets, int32_t* offsets, float* scores_or_null,
+                        int32_t* bucket_or_null, float* entropy_or_null, void* ws, size_t ws_bytes,
+                        void* stream);
+
+/*
+ * The whole pass on HOST buffers (pinned memory recommended): copies q_win, k, v, head_w and sens
+ * into `staging` (device memory, at least ckv_staging_bytes(), 256-byte aligned), runs
+ * ckv_compress, copies k_out, v_out, indices, budgets and offsets back, and synchronises the
+ * stream before returning.  Host tensors are dense ([Nu,H,W,d], [Nu,Hkv,L,d], head_w [Nu,H] or [H]
+ * by head_w_stride_unit, sens likewise); the strides in `shape` are ignored.
+ */
+size_t ckv_staging_bytes(const ckv_shape* shape, const ckv_params* params);
+ckv_status ckv_compress_host(const ckv_shape* shape, const ckv_params* params, const void* q_win_host,
+                             const void* k_host, const void* v_host, const float* head_w_host,
+                             const float* sens_host, void* k_out_host, void* v_out_host,
+                             int32_t* indices_host, int32_t* budgets_host, int32_t* offsets_host,
+                             void* staging, size_t staging_bytes, void* ws, size_t ws_bytes, void* stream);
+
+/* Synchronises `stream` and returns the status word device code wrote into `ws` (CKV_OK or
+ * CKV_ERR_TIMEOUT), or CKV_ERR_CUDA if the stream is in error. */
+ckv_status ckv_device_status(const void* ws, void* stream);
+
+/* Number of kernel launches this process has queued through the library so far. */
+int64_t ckv_kernel_launches(void);
+
+/* Host-only: the integer split of P prefix rows over hkv heads used by ckv_budget (demands >= 1,
+ * shares in [f, n], f*hkv <= P <= n*hkv), exposed so that it can be checked without a GPU.
+ * Returns 0 on success. */
+int ckv_allocate_rows_host(int hkv, int64_t n, int64_t f, int64_t P, const int64_t* demands, int64_t* out);
+
+const char* ckv_status_string(ckv_status status);
+int ckv_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CKV_H_ */

@@ -1,0 +1,234 @@
+"""Thin ctypes binding over the C ABI of ``libckv.so`` (see ``include/ckv.h``).
+
+Argument marshalling only: every step of the retention pass runs in the library's CUDA kernels.
+Functions carry the names of the C entry points and take torch CUDA tensors (device memory and
+streams are PyTorch's).  There is no fallback: a missing library or a non-zero status raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libckv.so")
+
+BF16, F32 = 0, 1
+POOL_NONE, POOL_MAX, POOL_AVG = 0, 1, 2
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
+
+
+class CkvError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: status {status} ({status_string(status)})")
+
+
+class ckv_shape(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("n_units", "n_q_heads", "n_kv_heads", "head_dim", "seq_len", "window",
+                                         "dtype", "reserved_")] + \
+               [(n, C.c_int64) for n in ("q_stride_unit", "q_stride_head", "q_stride_row",
+                                         "kv_stride_unit", "kv_stride_head", "kv_stride_tok")]
+
+
+class ckv_params(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("pool_kind", "pool_size", "budget_per_head", "floor_per_head",
+                                         "n_buckets", "bucket_override")] + \
+               [(n, C.c_int64) for n in ("head_w_stride_unit", "sens_stride_unit")]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads libckv.so; raises if it has not been built (``python -m paper_2602_08686_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2602_08686_b200.build` "
+                               "(there is no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        vp, sz, i32p, fp = C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p
+        shp, prm = C.POINTER(ckv_shape), C.POINTER(ckv_params)
+        L.ckv_workspace_bytes.restype = sz
+        L.ckv_workspace_bytes.argtypes = [shp, prm]
+        L.ckv_staging_bytes.restype = sz
+        L.ckv_staging_bytes.argtypes = [shp, prm]
+        L.ckv_score.argtypes = [shp, prm, vp, vp, fp, fp, fp, vp, sz, vp]
+        L.ckv_budget.argtypes = [shp, prm, fp, fp, fp, i32p, i32p, i32p, fp, vp, sz, vp]
+        L.ckv_select.argtypes = [shp, prm, fp, i32p, i32p, i32p, vp, sz, vp]
+        L.ckv_gather.argtypes = [shp, prm, vp, vp, i32p, i32p, vp, vp, vp]
+        L.ckv_compress.argtypes = [shp, prm, vp, vp, vp, fp, fp, vp, vp, i32p, i32p, i32p, fp, i32p, fp, vp, sz, vp]
+        L.ckv_compress_host.argtypes = [shp, prm, vp, vp, vp, fp, fp, vp, vp, i32p, i32p, i32p, vp, sz, vp, sz, vp]
+        L.ckv_device_status.argtypes = [vp, vp]
+        L.ckv_kernel_launches.restype = C.c_int64
+        L.ckv_status_string.restype = C.c_char_p
+        L.ckv_status_string.argtypes = [C.c_int]
+        L.ckv_allocate_rows_host.argtypes = [C.c_int, C.c_int64, C.c_int64, C.c_int64, vp, vp]
+        for name in ("ckv_score", "ckv_budget", "ckv_select", "ckv_gather", "ckv_compress", "ckv_compress_host",
+                     "ckv_device_status", "ckv_version", "ckv_allocate_rows_host"):
+            getattr(L, name).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().ckv_status_string(status).decode()
+
+
+def ckv_version() -> int:
+    return lib().ckv_version()
+
+
+def ckv_kernel_launches() -> int:
+    return int(lib().ckv_kernel_launches())
+
+
+@dataclass
+class Params:
+    pool_kind: int = POOL_MAX
+    pool_size: int = 7
+    budget_per_head: int = 512
+    floor_per_head: int = 1
+    n_buckets: int = 16
+    bucket_override: int = -1
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return BF16
+    if t.dtype == torch.float32:
+        return F32
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def make_shape(q: torch.Tensor, k: torch.Tensor) -> ckv_shape:
+    """Shape struct from q_win [Nu,H,W,d] and k [Nu,Hkv,L,d] (last dimension contiguous)."""
+    if q.dim() != 4 or k.dim() != 4 or q.stride(3) != 1 or k.stride(3) != 1:
+        raise ValueError("q_win and k must be 4-D with a contiguous last dimension")
+    Nu, H, W, d = q.shape
+    _, Hkv, L, _ = k.shape
+    return ckv_shape(Nu, H, Hkv, d, L, W, _dtype_code(k), 0, q.stride(0), q.stride(1), q.stride(2),
+                     k.stride(0), k.stride(1), k.stride(2))
+
+
+def make_params(p: Params, head_w: torch.Tensor | None, sens: torch.Tensor | None, H: int = 0) -> ckv_params:
+    hw_stride = 0 if head_w is None or head_w.dim() == 1 else head_w.stride(0)
+    se_stride = 0 if sens is None or sens.dim() == 1 else sens.stride(0)
+    return ckv_params(p.pool_kind, p.pool_size, p.budget_per_head, p.floor_per_head, p.n_buckets,
+                      p.bucket_override, hw_stride, se_stride)
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def _check(status: int, what: str):
+    if status != OK:
+        raise CkvError(status, what)
+
+
+def ckv_workspace_bytes(shape: ckv_shape, params: ckv_params) -> int:
+    return int(lib().ckv_workspace_bytes(C.byref(shape), C.byref(params)))
+
+
+def ckv_staging_bytes(shape: ckv_shape, params: ckv_params) -> int:
+    return int(lib().ckv_staging_bytes(C.byref(shape), C.byref(params)))
+
+
+def alloc_workspace(shape: ckv_shape, params: ckv_params, device) -> torch.Tensor:
+    nbytes = ckv_workspace_bytes(shape, params)
+    if nbytes == 0:
+        raise CkvError(ERR_INVALID_ARG, "ckv_workspace_bytes")
+    return torch.empty(nbytes, dtype=torch.uint8, device=device)
+
+
+def rows_per_unit(shape: ckv_shape, params: ckv_params) -> int:
+    return shape.n_kv_heads * min(params.budget_per_head, shape.seq_len)
+
+
+def ckv_score(shape, params, q_win, k, head_w, scores, colmass, ws, stream=None):
+    _check(lib().ckv_score(C.byref(shape), C.byref(params), _ptr(q_win), _ptr(k), _ptr(head_w), _ptr(scores),
+                           _ptr(colmass), _ptr(ws), ws.numel(), _stream(stream)), "ckv_score")
+
+
+def ckv_budget(shape, params, scores, colmass, sens, budgets, offsets, bucket, entropy, ws, stream=None):
+    _check(lib().ckv_budget(C.byref(shape), C.byref(params), _ptr(scores), _ptr(colmass), _ptr(sens), _ptr(budgets),
+                            _ptr(offsets), _ptr(bucket), _ptr(entropy), _ptr(ws), ws.numel(), _stream(stream)),
+           "ckv_budget")
+
+
+def ckv_select(shape, params, scores, budgets, offsets, indices, ws, stream=None):
+    _check(lib().ckv_select(C.byref(shape), C.byref(params), _ptr(scores), _ptr(budgets), _ptr(offsets),
+                            _ptr(indices), _ptr(ws), ws.numel(), _stream(stream)), "ckv_select")
+
+
+def ckv_gather(shape, params, k, v, indices, offsets, k_out, v_out, stream=None):
+    _check(lib().ckv_gather(C.byref(shape), C.byref(params), _ptr(k), _ptr(v), _ptr(indices), _ptr(offsets),
+                            _ptr(k_out), _ptr(v_out), _stream(stream)), "ckv_gather")
+
+
+def ckv_compress(shape, params, q_win, k, v, head_w, sens, k_out, v_out, indices, budgets, offsets, ws,
+                 scores=None, bucket=None, entropy=None, stream=None):
+    _check(lib().ckv_compress(C.byref(shape), C.byref(params), _ptr(q_win), _ptr(k), _ptr(v), _ptr(head_w),
+                              _ptr(sens), _ptr(k_out), _ptr(v_out), _ptr(indices), _ptr(budgets), _ptr(offsets),
+                              _ptr(scores), _ptr(bucket), _ptr(entropy), _ptr(ws), ws.numel(), _stream(stream)),
+           "ckv_compress")
+
+
+def ckv_compress_host(shape, params, q_win, k, v, head_w, sens, k_out, v_out, indices, budgets, offsets,
+                      staging, ws, stream=None):
+    """All tensor arguments except ``staging`` and ``ws`` are HOST tensors (pinned memory recommended)."""
+    _check(lib().ckv_compress_host(C.byref(shape), C.byref(params), _ptr(q_win), _ptr(k), _ptr(v), _ptr(head_w),
+                                   _ptr(sens), _ptr(k_out), _ptr(v_out), _ptr(indices), _ptr(budgets),
+                                   _ptr(offsets), _ptr(staging), staging.numel(), _ptr(ws), ws.numel(),
+                                   _stream(stream)), "ckv_compress_host")
+
+
+def ckv_device_status(ws, stream=None) -> int:
+    return int(lib().ckv_device_status(_ptr(ws), _stream(stream)))
+
+
+def ckv_allocate_rows_host(n: int, f: int, P: int, demands) -> list[int]:
+    """Host-side run of the integer budget split used by ckv_budget (no GPU needed)."""
+    hkv = len(demands)
+    dem = (C.c_int64 * hkv)(*[int(x) for x in demands])
+    out = (C.c_int64 * hkv)()
+    rc = lib().ckv_allocate_rows_host(hkv, n, f, P, dem, out)
+    if rc:
+        raise ValueError(f"ckv_allocate_rows_host failed with {rc}")
+    return list(out)
+
+
+# ------------------------------------------------------------------------------------ convenience
+def compress(q_win, k, v, head_w, sens, p: Params, want_scores: bool = False, ws=None, stream=None):
+    """Allocates the outputs and the work space with torch and runs ckv_compress."""
+    shape = make_shape(q_win, k)
+    params = make_params(p, head_w, sens)
+    dev = k.device
+    Nu, Hkv = shape.n_units, shape.n_kv_heads
+    rows = rows_per_unit(shape, params)
+    out = dict(
+        k_out=torch.empty(Nu, rows, shape.head_dim, dtype=k.dtype, device=dev),
+        v_out=torch.empty(Nu, rows, shape.head_dim, dtype=v.dtype, device=dev),
+        indices=torch.empty(Nu, rows, dtype=torch.int32, device=dev),
+        budgets=torch.empty(Nu, Hkv, dtype=torch.int32, device=dev),
+        offsets=torch.empty(Nu, Hkv + 1, dtype=torch.int32, device=dev),
+        bucket=torch.empty(Nu, dtype=torch.int32, device=dev),
+        entropy=torch.empty(Nu, dtype=torch.float32, device=dev),
+        scores=torch.empty(Nu, Hkv, shape.seq_len - shape.window, dtype=torch.float32, device=dev)
+        if want_scores else None,
+    )
+    ws = alloc_workspace(shape, params, dev) if ws is None else ws
+    ckv_compress(shape, params, q_win, k, v, head_w, sens, out["k_out"], out["v_out"], out["indices"],
+                 out["budgets"], out["offsets"], ws, scores=out["scores"], bucket=out["bucket"],
+                 entropy=out["entropy"], stream=stream)
+    out["ws"] = ws
+    return out

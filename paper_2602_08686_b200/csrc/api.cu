@@ -1,0 +1,298 @@
+// Host side of the C ABI: argument validation, work-space layout and the launch sequences.
+#include <atomic>
+#include <cstring>
+
+#include "ckv_common.cuh"
+
+namespace ckv {
+
+static std::atomic<int64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+static size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+WsLayout ws_layout(const ckv_shape& s, const ckv_params&) {
+  WsLayout w{};
+  const size_t Nu = s.n_units, H = s.n_q_heads, Hkv = s.n_kv_heads, L = s.seq_len, W = s.window;
+  const size_t n = L - W;
+  w.nblk = (int)((L + kPlainKeysPerBlock - 1) / kPlainKeysPerBlock);
+  size_t o = 0;
+  w.status = o, o += 256;
+  w.csum = o, o = align_up(o + Nu * H * L * sizeof(float));
+  w.part = o, o = align_up(o + Nu * H * W * (size_t)w.nblk * sizeof(float2));
+  w.stat = o, o = align_up(o + Nu * H * W * sizeof(float2));
+  w.colmass = o, o = align_up(o + Nu * L * sizeof(float));
+  w.scores = o, o = align_up(o + Nu * Hkv * (n ? n : 1) * sizeof(float));
+  w.bucket = o, o = align_up(o + Nu * sizeof(int32_t));
+  w.entropy = o, o = align_up(o + Nu * sizeof(float));
+  w.total = o;
+  return w;
+}
+
+static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+static ckv_status check_shape(const ckv_shape* s) {
+  if (!s) return CKV_ERR_INVALID_ARG;
+  if (s->n_units < 1 || s->n_q_heads < 1 || s->n_kv_heads < 1 || s->seq_len < 1 || s->window < 1)
+    return CKV_ERR_INVALID_ARG;
+  if (s->n_q_heads % s->n_kv_heads) return CKV_ERR_INVALID_ARG;
+  if (s->window > s->seq_len) return CKV_ERR_INVALID_ARG;
+  if (s->dtype != CKV_BF16 && s->dtype != CKV_F32) return CKV_ERR_INVALID_ARG;
+  if (s->head_dim != kHeadDim || s->window > kMaxWindow || s->n_kv_heads > kMaxKvHeads) return CKV_ERR_UNSUPPORTED;
+  if (s->n_units > 65535 || s->n_q_heads > 65535) return CKV_ERR_UNSUPPORTED;
+  if (s->seq_len > (1 << 20)) return CKV_ERR_UNSUPPORTED;
+  const int64_t esz = s->dtype == CKV_BF16 ? 2 : 4;
+  const int64_t strides[6] = {s->q_stride_unit, s->q_stride_head,  s->q_stride_row,
+                              s->kv_stride_unit, s->kv_stride_head, s->kv_stride_tok};
+  for (int64_t st : strides)
+    if (st < 0 || (st * esz) % 16) return CKV_ERR_INVALID_ARG;
+  if (s->q_stride_row < kHeadDim || s->kv_stride_tok < kHeadDim) return CKV_ERR_INVALID_ARG;
+  return CKV_OK;
+}
+
+static ckv_status check_params(const ckv_shape* s, const ckv_params* p) {
+  if (!p) return CKV_ERR_INVALID_ARG;
+  if (p->pool_kind < CKV_POOL_NONE || p->pool_kind > CKV_POOL_AVG) return CKV_ERR_INVALID_ARG;
+  if (p->pool_size < 1 || p->pool_size > 15 || (p->pool_size & 1) == 0) return CKV_ERR_INVALID_ARG;
+  if (p->budget_per_head < 1 || p->floor_per_head < 0 || p->n_buckets < 1) return CKV_ERR_INVALID_ARG;
+  if (p->bucket_override < -1 || p->bucket_override >= p->n_buckets) return CKV_ERR_INVALID_ARG;
+  if (p->head_w_stride_unit < 0 || p->sens_stride_unit < 0) return CKV_ERR_INVALID_ARG;
+  if (p->budget_per_head < s->seq_len) {
+    if (p->budget_per_head < s->window) return CKV_ERR_INVALID_ARG;
+    if (p->floor_per_head > p->budget_per_head - s->window) return CKV_ERR_INVALID_ARG;
+  }
+  return CKV_OK;
+}
+
+static ckv_status check_ws(const ckv_shape* s, const ckv_params* p, const void* ws, size_t ws_bytes) {
+  if (!ws || !aligned(ws, 256) || ws_bytes < ws_layout(*s, *p).total) return CKV_ERR_WORKSPACE;
+  return CKV_OK;
+}
+
+static bool all_aligned16(std::initializer_list<const void*> ps) {
+  for (const void* p : ps)
+    if (!p || !aligned(p, 16)) return false;
+  return true;
+}
+static bool all_aligned4(std::initializer_list<const void*> ps) {
+  for (const void* p : ps)
+    if (!p || !aligned(p, 4)) return false;
+  return true;
+}
+
+#define CKV_TRY(expr)                  \
+  do {                                 \
+    ckv_status st__ = (expr);          \
+    if (st__ != CKV_OK) return st__;   \
+  } while (0)
+#define CKV_CUDA(expr)                               \
+  do {                                               \
+    if ((expr) != cudaSuccess) return CKV_ERR_CUDA;  \
+  } while (0)
+
+static ckv_status score_impl(const ckv_shape& s, const ckv_params& p, const void* q, const void* k,
+                             const float* head_w, float* scores, float* colmass, char* ws, cudaStream_t st) {
+  const WsLayout w = ws_layout(s, p);
+  CKV_CUDA(cudaMemsetAsync(ws + w.status, 0, 256, st));
+  float* csum = reinterpret_cast<float*>(ws + w.csum);
+  CKV_CUDA(launch_score_plain(s, q, k, csum, reinterpret_cast<float2*>(ws + w.part),
+                              reinterpret_cast<float2*>(ws + w.stat), w.nblk, st));
+  CKV_CUDA(launch_epilogue(s, p, csum, head_w, scores, colmass, st));
+  return CKV_OK;
+}
+
+}  // namespace ckv
+
+using namespace ckv;
+
+#pragma GCC visibility push(default)
+extern "C" {
+
+size_t ckv_workspace_bytes(const ckv_shape* shape, const ckv_params* params) {
+  if (check_shape(shape) != CKV_OK || check_params(shape, params) != CKV_OK) return 0;
+  return ws_layout(*shape, *params).total;
+}
+
+ckv_status ckv_score(const ckv_shape* shape, const ckv_params* params, const void* q_win, const void* k,
+                     const float* head_w, float* scores, float* colmass, void* ws, size_t ws_bytes, void* stream) {
+  CKV_TRY(check_shape(shape));
+  CKV_TRY(check_params(shape, params));
+  if (!all_aligned16({q_win, k}) || !all_aligned4({head_w, scores, colmass})) return CKV_ERR_INVALID_ARG;
+  CKV_TRY(check_ws(shape, params, ws, ws_bytes));
+  return score_impl(*shape, *params, q_win, k, head_w, scores, colmass, (char*)ws, (cudaStream_t)stream);
+}
+
+ckv_status ckv_budget(const ckv_shape* shape, const ckv_params* params, const float* scores, const float* colmass,
+                      const float* sens, int32_t* budgets, int32_t* offsets, int32_t* bucket, float* entropy,
+                      void* ws, size_t ws_bytes, void* stream) {
+  CKV_TRY(check_shape(shape));
+  CKV_TRY(check_params(shape, params));
+  if (!all_aligned4({scores, colmass, sens, budgets, offsets, bucket, entropy})) return CKV_ERR_INVALID_ARG;
+  CKV_TRY(check_ws(shape, params, ws, ws_bytes));
+  CKV_CUDA(launch_budget(*shape, *params, scores, colmass, sens, budgets, offsets, bucket, entropy,
+                         (cudaStream_t)stream));
+  return CKV_OK;
+}
+
+ckv_status ckv_select(const ckv_shape* shape, const ckv_params* params, const float* scores, const int32_t* budgets,
+                      const int32_t* offsets, int32_t* indices, void* ws, size_t ws_bytes, void* stream) {
+  CKV_TRY(check_shape(shape));
+  CKV_TRY(check_params(shape, params));
+  if (!all_aligned4({scores, budgets, offsets, indices})) return CKV_ERR_INVALID_ARG;
+  CKV_TRY(check_ws(shape, params, ws, ws_bytes));
+  CKV_CUDA(launch_select(*shape, *params, scores, budgets, offsets, indices, (cudaStream_t)stream));
+  return CKV_OK;
+}
+
+ckv_status ckv_gather(const ckv_shape* shape, const ckv_params* params, const void* k, const void* v,
+                      const int32_t* indices, const int32_t* offsets, void* k_out, void* v_out, void* stream) {
+  CKV_TRY(check_shape(shape));
+  CKV_TRY(check_params(shape, params));
+  if (!all_aligned16({k, v, k_out, v_out}) || !all_aligned4({indices, offsets})) return CKV_ERR_INVALID_ARG;
+  CKV_CUDA(launch_gather(*shape, *params, k, v, indices, offsets, k_out, v_out, (cudaStream_t)stream));
+  return CKV_OK;
+}
+
+ckv_status ckv_compress(const ckv_shape* shape, const ckv_params* params, const void* q_win, const void* k,
+                        const void* v, const float* head_w, const float* sens, void* k_out, void* v_out,
+                        int32_t* indices, int32_t* budgets, int32_t* offsets, float* scores_or_null,
+                        int32_t* bucket_or_null, float* entropy_or_null, void* ws, size_t ws_bytes, void* stream) {
+  CKV_TRY(check_shape(shape));
+  CKV_TRY(check_params(shape, params));
+  if (!all_aligned16({q_win, k, v, k_out, v_out}) || !all_aligned4({head_w, sens, indices, budgets, offsets}))
+    return CKV_ERR_INVALID_ARG;
+  if ((scores_or_null && !aligned(scores_or_null, 4)) || (bucket_or_null && !aligned(bucket_or_null, 4)) ||
+      (entropy_or_null && !aligned(entropy_or_null, 4)))
+    return CKV_ERR_INVALID_ARG;
+  CKV_TRY(check_ws(shape, params, ws, ws_bytes));
+  const WsLayout w = ws_layout(*shape, *params);
+  char* base = (char*)ws;
+  cudaStream_t st = (cudaStream_t)stream;
+  float* scores = scores_or_null ? scores_or_null : reinterpret_cast<float*>(base + w.scores);
+  float* colmass = reinterpret_cast<float*>(base + w.colmass);
+  int32_t* bucket = bucket_or_null ? bucket_or_null : reinterpret_cast<int32_t*>(base + w.bucket);
+  float* entropy = entropy_or_null ? entropy_or_null : reinterpret_cast<float*>(base + w.entropy);
+  CKV_TRY(score_impl(*shape, *params, q_win, k, head_w, scores, colmass, base, st));
+  CKV_CUDA(launch_budget(*shape, *params, scores, colmass, sens, budgets, offsets, bucket, entropy, st));
+  CKV_CUDA(launch_select(*shape, *params, scores, budgets, offsets, indices, st));
+  CKV_CUDA(launch_gather(*shape, *params, k, v, indices, offsets, k_out, v_out, st));
+  return CKV_OK;
+}
+
+// staging sections: q | k | v | head_w | sens | k_out | v_out | indices | budgets | offsets
+struct Staging {
+  size_t q, k, v, head_w, sens, k_out, v_out, indices, budgets, offsets, total;
+  size_t q_b, kv_b, hw_b, sens_b, out_b, idx_b, bud_b, off_b;
+};
+static Staging staging_layout(const ckv_shape& s, const ckv_params& p) {
+  Staging g{};
+  const size_t esz = s.dtype == CKV_BF16 ? 2 : 4;
+  const size_t Nu = s.n_units, H = s.n_q_heads, Hkv = s.n_kv_heads, L = s.seq_len, W = s.window, d = s.head_dim;
+  const size_t rows = Hkv * (size_t)(p.budget_per_head < s.seq_len ? p.budget_per_head : s.seq_len);
+  g.q_b = Nu * H * W * d * esz;
+  g.kv_b = Nu * Hkv * L * d * esz;
+  g.hw_b = (p.head_w_stride_unit ? Nu : 1) * H * sizeof(float);
+  g.sens_b = (p.sens_stride_unit ? Nu : 1) * (size_t)p.n_buckets * sizeof(float);
+  g.out_b = Nu * rows * d * esz;
+  g.idx_b = Nu * rows * sizeof(int32_t);
+  g.bud_b = Nu * Hkv * sizeof(int32_t);
+  g.off_b = Nu * (Hkv + 1) * sizeof(int32_t);
+  size_t o = 0;
+  g.q = o, o = align_up(o + g.q_b);
+  g.k = o, o = align_up(o + g.kv_b);
+  g.v = o, o = align_up(o + g.kv_b);
+  g.head_w = o, o = align_up(o + g.hw_b);
+  g.sens = o, o = align_up(o + g.sens_b);
+  g.k_out = o, o = align_up(o + g.out_b);
+  g.v_out = o, o = align_up(o + g.out_b);
+  g.indices = o, o = align_up(o + g.idx_b);
+  g.budgets = o, o = align_up(o + g.bud_b);
+  g.offsets = o, o = align_up(o + g.off_b);
+  g.total = o;
+  return g;
+}
+
+size_t ckv_staging_bytes(const ckv_shape* shape, const ckv_params* params) {
+  if (check_shape(shape) != CKV_OK || check_params(shape, params) != CKV_OK) return 0;
+  return staging_layout(*shape, *params).total;
+}
+
+ckv_status ckv_compress_host(const ckv_shape* shape, const ckv_params* params, const void* q_win_host,
+                             const void* k_host, const void* v_host, const float* head_w_host,
+                             const float* sens_host, void* k_out_host, void* v_out_host, int32_t* indices_host,
+                             int32_t* budgets_host, int32_t* offsets_host, void* staging, size_t staging_bytes,
+                             void* ws, size_t ws_bytes, void* stream) {
+  CKV_TRY(check_shape(shape));
+  CKV_TRY(check_params(shape, params));
+  if (!q_win_host || !k_host || !v_host || !head_w_host || !sens_host || !k_out_host || !v_out_host ||
+      !indices_host || !budgets_host || !offsets_host)
+    return CKV_ERR_INVALID_ARG;
+  const Staging g = staging_layout(*shape, *params);
+  if (!staging || !aligned(staging, 256) || staging_bytes < g.total) return CKV_ERR_WORKSPACE;
+  CKV_TRY(check_ws(shape, params, ws, ws_bytes));
+  ckv_shape s = *shape;  // dense device copies
+  s.q_stride_row = s.head_dim;
+  s.q_stride_head = (int64_t)s.window * s.head_dim;
+  s.q_stride_unit = (int64_t)s.n_q_heads * s.q_stride_head;
+  s.kv_stride_tok = s.head_dim;
+  s.kv_stride_head = (int64_t)s.seq_len * s.head_dim;
+  s.kv_stride_unit = (int64_t)s.n_kv_heads * s.kv_stride_head;
+  ckv_params p = *params;
+  p.head_w_stride_unit = params->head_w_stride_unit ? s.n_q_heads : 0;
+  p.sens_stride_unit = params->sens_stride_unit ? params->n_buckets : 0;
+  char* d = (char*)staging;
+  cudaStream_t st = (cudaStream_t)stream;
+  CKV_CUDA(cudaMemcpyAsync(d + g.q, q_win_host, g.q_b, cudaMemcpyHostToDevice, st));
+  CKV_CUDA(cudaMemcpyAsync(d + g.k, k_host, g.kv_b, cudaMemcpyHostToDevice, st));
+  CKV_CUDA(cudaMemcpyAsync(d + g.v, v_host, g.kv_b, cudaMemcpyHostToDevice, st));
+  CKV_CUDA(cudaMemcpyAsync(d + g.head_w, head_w_host, g.hw_b, cudaMemcpyHostToDevice, st));
+  CKV_CUDA(cudaMemcpyAsync(d + g.sens, sens_host, g.sens_b, cudaMemcpyHostToDevice, st));
+  CKV_TRY(ckv_compress(&s, &p, d + g.q, d + g.k, d + g.v, (const float*)(d + g.head_w), (const float*)(d + g.sens),
+                       d + g.k_out, d + g.v_out, (int32_t*)(d + g.indices), (int32_t*)(d + g.budgets),
+                       (int32_t*)(d + g.offsets), nullptr, nullptr, nullptr, ws, ws_bytes, stream));
+  CKV_CUDA(cudaMemcpyAsync(k_out_host, d + g.k_out, g.out_b, cudaMemcpyDeviceToHost, st));
+  CKV_CUDA(cudaMemcpyAsync(v_out_host, d + g.v_out, g.out_b, cudaMemcpyDeviceToHost, st));
+  CKV_CUDA(cudaMemcpyAsync(indices_host, d + g.indices, g.idx_b, cudaMemcpyDeviceToHost, st));
+  CKV_CUDA(cudaMemcpyAsync(budgets_host, d + g.budgets, g.bud_b, cudaMemcpyDeviceToHost, st));
+  CKV_CUDA(cudaMemcpyAsync(offsets_host, d + g.offsets, g.off_b, cudaMemcpyDeviceToHost, st));
+  CKV_CUDA(cudaStreamSynchronize(st));
+  return CKV_OK;
+}
+
+ckv_status ckv_device_status(const void* ws, void* stream) {
+  if (!ws) return CKV_ERR_WORKSPACE;
+  int32_t word = 0;
+  if (cudaMemcpyAsync(&word, ws, sizeof(word), cudaMemcpyDeviceToHost, (cudaStream_t)stream) != cudaSuccess)
+    return CKV_ERR_CUDA;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return CKV_ERR_CUDA;
+  return word == 0 ? CKV_OK : CKV_ERR_TIMEOUT;
+}
+
+int64_t ckv_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* ckv_status_string(ckv_status status) {
+  switch (status) {
+    case CKV_OK: return "ok";
+    case CKV_ERR_INVALID_ARG: return "invalid argument";
+    case CKV_ERR_UNSUPPORTED: return "unsupported shape";
+    case CKV_ERR_WORKSPACE: return "work space missing, misaligned or too small";
+    case CKV_ERR_CUDA: return "CUDA error";
+    case CKV_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+int ckv_version(void) { return 100; }
+
+// Host-only check of the budget split used by the device code (same source, compiled for the host).
+int ckv_allocate_rows_host(int hkv, int64_t n, int64_t f, int64_t P, const int64_t* demands, int64_t* out) {
+  if (hkv < 1 || hkv > kMaxKvHeads) return 1;
+  long long dem[kMaxKvHeads], e[kMaxKvHeads];
+  for (int g = 0; g < hkv; ++g) dem[g] = demands[g];
+  if (!allocate_rows(hkv, n, f, P, dem, e)) return 2;
+  for (int g = 0; g < hkv; ++g) out[g] = e[g];
+  return 0;
+}
+
+}  // extern "C"
+#pragma GCC visibility pop

@@ -1,0 +1,124 @@
+// Internal declarations shared by the translation units of libckv (not part of the C ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/ckv.h"
+
+namespace ckv {
+
+constexpr int kHeadDim = 128;
+constexpr int kMaxWindow = 64;
+constexpr int kMaxKvHeads = 64;
+constexpr int kPlainKeysPerBlock = 256;  // keys per CTA in the plain (SIMT) score kernels
+
+// log2(e): the softmax is evaluated in base 2, x = (q.k) * log2(e) / sqrt(d)
+constexpr float kLog2e = 1.4426950408889634f;
+
+// Work-space sections (byte offsets from the 256-byte aligned base).
+struct WsLayout {
+  size_t status;   // 64 x int32: [0] device status word, the rest scheduler counters
+  size_t csum;     // float [Nu, H, L]        c_h[t]
+  size_t part;     // float2 [Nu, H, W, nblk] per-block (max, sum) of the row statistics
+  size_t stat;     // float2 [Nu, H, W]       (row max, row max + log2 row sum), base-2 domain
+  size_t colmass;  // float [Nu, L]           used when the caller passes no buffer
+  size_t scores;   // float [Nu, Hkv, n]      likewise
+  size_t bucket;   // int32 [Nu]
+  size_t entropy;  // float [Nu]
+  size_t total;
+  int nblk;
+};
+
+WsLayout ws_layout(const ckv_shape& s, const ckv_params& p);
+
+void count_launch(int n = 1);
+
+// Launchers; each returns cudaGetLastError() after queuing its kernels.
+cudaError_t launch_score_plain(const ckv_shape& s, const void* q, const void* k, float* csum, float2* part,
+                               float2* stat, int nblk, cudaStream_t st);
+cudaError_t launch_epilogue(const ckv_shape& s, const ckv_params& p, const float* csum, const float* head_w,
+                            float* scores, float* colmass, cudaStream_t st);
+cudaError_t launch_budget(const ckv_shape& s, const ckv_params& p, const float* scores, const float* colmass,
+                          const float* sens, int32_t* budgets, int32_t* offsets, int32_t* bucket, float* entropy,
+                          cudaStream_t st);
+cudaError_t launch_select(const ckv_shape& s, const ckv_params& p, const float* scores, const int32_t* budgets,
+                          const int32_t* offsets, int32_t* indices, cudaStream_t st);
+cudaError_t launch_gather(const ckv_shape& s, const ckv_params& p, const void* k, const void* v,
+                          const int32_t* indices, const int32_t* offsets, void* k_out, void* v_out,
+                          cudaStream_t st);
+
+// ---------------------------------------------------------------------------------------------
+// Split P prefix rows over `hkv` heads in proportion to demands dem[g] >= 1 with every share held
+// in [f, n] (the clamp of the per-head budgets to the unit's total).  Heads are visited in order of
+// demand; because the clamp is monotone in the demand, the heads pinned at the floor are the `a`
+// smallest demands and the heads pinned at the cap the `b` largest.  All (a, b) are tried until
+// the water level R / D of the unpinned heads is consistent with that split.  Shares of unpinned
+// heads are rounded down and the remainder goes to the largest fractional parts, ties to the
+// lowest head index.  Pure integer arithmetic (products stay below 2^62 for n <= 2^20, hkv <= 64).
+// Returns false only if the arguments violate f*hkv <= P <= n*hkv.
+__host__ __device__ inline bool allocate_rows(int hkv, long long n, long long f, long long P, const long long* dem,
+                                              long long* e) {
+  int order[kMaxKvHeads];
+  for (int g = 0; g < hkv; ++g) order[g] = g;
+  for (int i = 1; i < hkv; ++i) {  // stable insertion sort by demand
+    int x = order[i], j = i - 1;
+    while (j >= 0 && dem[order[j]] > dem[x]) {
+      order[j + 1] = order[j];
+      --j;
+    }
+    order[j + 1] = x;
+  }
+  long long total = 0;
+  for (int g = 0; g < hkv; ++g) total += dem[g];
+  long long low_sum = 0;  // sum of the a smallest demands
+  for (int a = 0; a <= hkv; ++a) {
+    if (a > 0) low_sum += dem[order[a - 1]];
+    long long high_sum = 0;
+    for (int b = 0; a + b <= hkv; ++b) {
+      if (b > 0) high_sum += dem[order[hkv - b]];
+      const long long R = P - a * f - b * n;
+      const long long D = total - low_sum - high_sum;
+      const int mid = hkv - a - b;
+      bool ok;
+      if (mid == 0) {
+        ok = (R == 0);
+      } else {
+        const long long dmin = dem[order[a]], dmax = dem[order[hkv - b - 1]];
+        ok = R >= 0 && R * dmin >= f * D && R * dmax <= n * D;
+        if (ok && a > 0) ok = R * dem[order[a - 1]] <= f * D;
+        if (ok && b > 0) ok = R * dem[order[hkv - b]] >= n * D;
+      }
+      if (!ok) continue;
+      long long rem[kMaxKvHeads];
+      long long given = 0;
+      for (int r = 0; r < hkv; ++r) {
+        const int g = order[r];
+        if (r < a) {
+          e[g] = f;
+          rem[g] = 0;
+        } else if (r >= hkv - b) {
+          e[g] = n;
+          rem[g] = 0;
+        } else {
+          e[g] = (R * dem[g]) / D;
+          rem[g] = (R * dem[g]) % D;
+          given += e[g];
+        }
+      }
+      long long left = mid > 0 ? R - given : 0;
+      while (left > 0) {
+        int best = -1;
+        for (int g = 0; g < hkv; ++g)
+          if (rem[g] > 0 && (best < 0 || rem[g] > rem[best])) best = g;
+        if (best < 0) return false;
+        e[best] += 1;
+        rem[best] = 0;
+        --left;
+      }
+      return true;
+    }
+  }
+  return false;
+}
+
+}  // namespace ckv

@@ -1,0 +1,351 @@
+"""GPU parity: the CUDA library (through its C ABI) against the fp64 oracle on the same seeded inputs.
+
+Protocol (discrete stages never inherit float noise):
+  1. scores: max relative error <= 1e-3 over every prefix position; entropy abs error <= 1e-4.
+  2. bucket: equal unless n_buckets * entropy / ln L is within 1e-4 of an integer.
+  3. ckv_budget fed the oracle's scores rounded to fp32 (both sides see identical bits): budgets and
+     offsets exactly equal.  In the fused path the GPU budgets equal the oracle's budget step run on
+     the GPU's own scores, exactly.
+  4. ckv_select on identical fp32 scores and budgets: identical indices.  Against the oracle's own
+     fp64 scores the symmetric difference lies inside the near-tie band (1e-3 relative of the k-th score).
+  5. gather: bit-exact given the indices.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import Problem
+from paper_2602_08686_b200 import inputs as gen
+
+pytestmark = pytest.mark.gpu
+
+SCORE_RTOL = 1e-3          # spec tolerance on pooled, weighted scores
+TIE_BAND = 1e-3            # selection may differ only inside this relative band around the k-th score
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2602_08686_b200 import binding
+    binding.lib()
+    assert torch.cuda.is_available()
+    return binding
+
+
+def problem_of(cfg, Nu, **kw):
+    prob = Problem(Nu, cfg.n_q_heads, cfg.n_kv_heads, cfg.seq_len, cfg.window, head_dim=cfg.head_dim,
+                   dtype=oracle.BF16 if cfg.dtype == "bf16" else oracle.F32, pool_kind=cfg.pool_kind,
+                   pool_size=cfg.pool_size, budget_per_head=cfg.budget_per_head, floor_per_head=cfg.floor_per_head,
+                   n_buckets=cfg.n_buckets)
+    for k, v in kw.items():
+        setattr(prob, k, v)
+    return prob
+
+
+def params_of(B, prob):
+    return B.Params(pool_kind=prob.pool_kind, pool_size=prob.pool_size, budget_per_head=prob.budget_per_head,
+                    floor_per_head=prob.floor_per_head, n_buckets=prob.n_buckets,
+                    bucket_override=prob.bucket_override)
+
+
+def oracle_all(prob, b):
+    q, k, v, hw, sens = (gen.as_numpy(b[x]) for x in ("q", "k", "v", "head_w", "sens"))
+    scores, colmass = oracle.score(prob, q, k, hw)
+    bud = oracle.budget(prob, scores, colmass, sens)
+    idx = oracle.select(prob, scores, bud["budgets"], bud["offsets"])
+    return dict(scores=scores, colmass=colmass, idx=idx, **bud)
+
+
+def check_scores(gpu_scores, gpu_colmass, gpu_entropy, ref, prob):
+    s = gpu_scores.double().cpu().numpy()
+    rel = np.abs(s - ref["scores"]) / np.maximum(np.abs(ref["scores"]), 1e-20)
+    assert rel.max() <= SCORE_RTOL, f"score rel err {rel.max():.3e}"
+    cm = gpu_colmass.double().cpu().numpy()
+    np.testing.assert_allclose(cm, ref["colmass"], rtol=SCORE_RTOL, atol=1e-12)
+    assert np.abs(gpu_entropy.double().cpu().numpy() - ref["entropy"]).max() <= 1e-4
+    return rel.max()
+
+
+def check_bucket(gpu_bucket, ref, prob):
+    hn = ref["entropy"] / math.log(prob.seq_len) * prob.n_buckets
+    near = np.abs(hn - np.round(hn)) < 1e-4
+    got = gpu_bucket.cpu().numpy()
+    assert ((got == ref["bucket"]) | near).all()
+
+
+def check_selection_against_oracle(gpu_idx, gpu_budgets, gpu_offsets, ref, prob):
+    """Same budgets: the index sets may differ only inside the near-tie band of the oracle's scores."""
+    W, n = prob.window, prob.n
+    for u in range(prob.n_units):
+        if not (gpu_budgets[u] == ref["budgets"][u]).all():
+            continue  # different budgets (a score within the band of tau): compared elsewhere
+        for g in range(prob.n_kv_heads):
+            a = set(gpu_idx[u, gpu_offsets[u, g]: gpu_offsets[u, g + 1]].tolist())
+            r = set(ref["idx"][u, ref["offsets"][u, g]: ref["offsets"][u, g + 1]].tolist())
+            diff = a ^ r
+            if not diff:
+                continue
+            e = ref["budgets"][u, g] - W
+            sc = ref["scores"][u, g]
+            kth = np.sort(sc)[::-1][e - 1]
+            for t in diff:
+                assert t < n and abs(sc[t] - kth) <= TIE_BAND * abs(kth), (u, g, t, sc[t], kth)
+
+
+def check_structure(idx, budgets, offsets, prob, needles=None, cfg=None):
+    L, W, n, Hkv = prob.seq_len, prob.window, prob.n, prob.n_kv_heads
+    rows = Hkv * prob.rows_per_head
+    assert (budgets.sum(1) == rows).all()
+    assert (offsets[:, 0] == 0).all() and (np.diff(offsets, axis=1) == budgets).all()
+    for u in range(prob.n_units):
+        for g in range(Hkv):
+            s = idx[u, offsets[u, g]: offsets[u, g + 1]]
+            assert (np.diff(s) > 0).all() and s[0] >= 0 and s[-1] == L - 1
+            assert (s[-W:] == np.arange(n, L)).all()
+            if prob.budget_per_head < L:
+                assert budgets[u, g] - W >= prob.floor_per_head
+
+
+def check_gather(k, v, k_out, v_out, idx, offsets, prob):
+    kn, vn = gen.as_numpy(k), gen.as_numpy(v)
+    ko, vo = gen.as_numpy(k_out), gen.as_numpy(v_out)
+    for u in range(prob.n_units):
+        for g in range(prob.n_kv_heads):
+            sl = slice(offsets[u, g], offsets[u, g + 1])
+            np.testing.assert_array_equal(ko[u, sl], kn[u, g, idx[u, sl]])
+            np.testing.assert_array_equal(vo[u, sl], vn[u, g, idx[u, sl]])
+
+
+def run_case(B, cfg, units=None, **prob_kw):
+    """Staged and fused GPU runs of one case against the oracle; returns the worst score error."""
+    b_cpu = gen.make_batch(cfg, "cpu", units)
+    Nu = len(b_cpu["units"])
+    prob = problem_of(cfg, Nu, **prob_kw)
+    ref = oracle_all(prob, b_cpu)
+    b = {k: (v.cuda() if torch.is_tensor(v) else v) for k, v in b_cpu.items()}
+    P = params_of(B, prob)
+    shape = B.make_shape(b["q"], b["k"])
+    params = B.make_params(P, b["head_w"], b["sens"])
+    ws = B.alloc_workspace(shape, params, "cuda")
+    n, Hkv, L = prob.n, prob.n_kv_heads, prob.seq_len
+    rows = B.rows_per_unit(shape, params)
+    dev = "cuda"
+
+    # ---- staged path -------------------------------------------------------------------------
+    scores = torch.full((Nu, Hkv, n), float("nan"), device=dev)
+    colmass = torch.full((Nu, L), float("nan"), device=dev)
+    B.ckv_score(shape, params, b["q"], b["k"], b["head_w"], scores, colmass, ws)
+    budgets = torch.zeros(Nu, Hkv, dtype=torch.int32, device=dev)
+    offsets = torch.zeros(Nu, Hkv + 1, dtype=torch.int32, device=dev)
+    bucket = torch.zeros(Nu, dtype=torch.int32, device=dev)
+    entropy = torch.zeros(Nu, device=dev)
+    B.ckv_budget(shape, params, scores, colmass, b["sens"], budgets, offsets, bucket, entropy, ws)
+    err = check_scores(scores, colmass, entropy, ref, prob)
+    check_bucket(bucket, ref, prob)
+
+    # (3) budget on identical bits: the oracle's scores rounded to fp32, the oracle's bucket forced
+    s32 = torch.from_numpy(ref["scores"]).float()
+    cm32 = torch.from_numpy(ref["colmass"]).float()
+    for u_bucket in sorted(set(ref["bucket"].tolist())):
+        sel = [u for u in range(Nu) if ref["bucket"][u] == u_bucket]
+        prob_b = problem_of(cfg, Nu, **{**prob_kw, "bucket_override": int(u_bucket)})
+        ref_b = oracle.budget(prob_b, s32.double().numpy(), cm32.double().numpy(), gen.as_numpy(b_cpu["sens"]))
+        params_b = B.make_params(params_of(B, prob_b), b["head_w"], b["sens"])
+        bud_g = torch.zeros_like(budgets)
+        off_g = torch.zeros_like(offsets)
+        B.ckv_budget(shape, params_b, s32.cuda(), cm32.cuda(), b["sens"], bud_g, off_g, bucket.clone(),
+                     entropy.clone(), ws)
+        assert (bud_g.cpu().numpy()[sel] == ref_b["budgets"][sel]).all()
+        assert (off_g.cpu().numpy()[sel] == ref_b["offsets"][sel]).all()
+
+    # (4) select on identical bits
+    ref_bud = torch.from_numpy(ref["budgets"]).cuda()
+    ref_off = torch.from_numpy(ref["offsets"]).cuda()
+    idx_g = torch.full((Nu, rows), -1, dtype=torch.int32, device=dev)
+    B.ckv_select(shape, params, s32.cuda(), ref_bud, ref_off, idx_g, ws)
+    want = oracle.select(prob, s32.double().numpy(), ref["budgets"], ref["offsets"])
+    np.testing.assert_array_equal(idx_g.cpu().numpy(), want)
+    # the GPU's own scores with the oracle's budgets: near-tie protocol
+    B.ckv_select(shape, params, scores, ref_bud, ref_off, idx_g, ws)
+    check_selection_against_oracle(idx_g.cpu().numpy(), ref["budgets"], ref["offsets"], ref, prob)
+
+    # (5) gather
+    k_out = torch.zeros(Nu, rows, prob.head_dim, dtype=b["k"].dtype, device=dev)
+    v_out = torch.zeros_like(k_out)
+    B.ckv_gather(shape, params, b["k"], b["v"], idx_g, ref_off, k_out, v_out)
+    check_gather(b_cpu["k"], b_cpu["v"], k_out, v_out, idx_g.cpu().numpy(), ref["offsets"], prob)
+
+    # ---- fused path --------------------------------------------------------------------------
+    out = B.compress(b["q"], b["k"], b["v"], b["head_w"], b["sens"], P, want_scores=True, ws=ws)
+    assert B.ckv_device_status(ws) == B.OK
+    assert torch.equal(out["scores"], scores)                       # deterministic, same kernels
+    gs = out["scores"].double().cpu().numpy()
+    # the oracle's budget step on the GPU's own scores, with the GPU's bucket: exact equality
+    gpu_budgets, gpu_offsets = out["budgets"].cpu().numpy(), out["offsets"].cpu().numpy()
+    gpu_bucket = out["bucket"].cpu().numpy()
+    for u in range(Nu):
+        prob_u = problem_of(cfg, 1, **{**prob_kw, "bucket_override": int(gpu_bucket[u])})
+        ref_u = oracle.budget(prob_u, gs[u:u + 1], colmass[u:u + 1].double().cpu().numpy(),
+                              gen.as_numpy(b_cpu["sens"]))
+        assert (ref_u["budgets"][0] == gpu_budgets[u]).all(), (u, ref_u["budgets"], gpu_budgets[u])
+    gpu_idx = out["indices"].cpu().numpy()
+    np.testing.assert_array_equal(gpu_idx, oracle.select(prob, gs, gpu_budgets, gpu_offsets))
+    check_structure(gpu_idx, gpu_budgets, gpu_offsets, prob)
+    check_selection_against_oracle(gpu_idx, gpu_budgets, gpu_offsets, ref, prob)
+    check_gather(b_cpu["k"], b_cpu["v"], out["k_out"], out["v_out"], gpu_idx, gpu_offsets, prob)
+    return err
+
+
+# ------------------------------------------------------------------------------------------ cases
+def test_config1_fp32_whole(B):
+    """Config 1 as specified: one layer, 8/2 heads, fp32, L 2048, W 32, MAX pool 7, B 512."""
+    run_case(B, gen.CONFIGS["c1"])
+
+
+@pytest.mark.parametrize("L", [4096, 4000, 1111])
+def test_llama_shape_small(B, L):
+    """Config 2's head layout at lengths that span several key tiles and leave a ragged tail."""
+    cfg = gen.shrink(gen.CONFIGS["c2"], n_layers=2, seq_len=L, budget_per_head=128, n_needles=8)
+    run_case(B, cfg)
+
+
+def test_heavy_tail_keys(B):
+    """Config 4's structure (Student-t key scales, stratified needles) at a length the oracle finishes."""
+    cfg = gen.shrink(gen.CONFIGS["c4"], n_layers=2, seq_len=8192, budget_per_head=128, n_needles=16)
+    run_case(B, cfg)
+
+
+@pytest.mark.parametrize("budget", [128, 512])
+def test_qwen_shape_L4096(B, budget):
+    """Config 5 at L 4096: GQA 7, W 64, AVG pool 5, floor 8, one low-reliability group per layer."""
+    cfg = gen.shrink(gen.c5_point(4096, budget), n_layers=2, batch=2)
+    run_case(B, cfg)
+
+
+@pytest.mark.parametrize("override", [0, 7, 15])
+def test_bucket_override(B, override):
+    cfg = gen.shrink(gen.CONFIGS["c2"], n_layers=1, n_q_heads=8, n_kv_heads=2, seq_len=1500, budget_per_head=96,
+                     n_needles=4)
+    run_case(B, cfg, bucket_override=override)
+
+
+@pytest.mark.parametrize("pool_kind,pool_size", [(0, 1), (1, 1), (1, 3), (1, 15), (2, 3), (2, 7), (2, 15)])
+def test_pooling_variants(B, pool_kind, pool_size):
+    cfg = gen.shrink(gen.CONFIGS["c2"], n_layers=1, n_q_heads=8, n_kv_heads=2, seq_len=1000, budget_per_head=80,
+                     n_needles=4, pool_kind=pool_kind, pool_size=pool_size)
+    run_case(B, cfg)
+
+
+@pytest.mark.parametrize("W,L,Bud", [(1, 300, 10), (8, 8, 8), (16, 40, 16), (32, 600, 700), (64, 64, 100),
+                                      (5, 261, 6), (32, 257, 33)])
+def test_degenerate_shapes(B, W, L, Bud):
+    """Window of one row, L == W (empty prefix), B == W (window only), B >= L (FullKV), tiny prefixes."""
+    cfg = gen.shrink(gen.CONFIGS["c2"], n_layers=2, n_q_heads=4, n_kv_heads=2, seq_len=L, window=W,
+                     budget_per_head=Bud, floor_per_head=0, n_needles=0, pool_size=3)
+    b_cpu = gen.make_batch(cfg, "cpu") if L - W > 8 else None
+    if b_cpu is None:
+        # the needle planter needs a prefix; draw plain random tensors instead
+        g = torch.Generator().manual_seed(L * 100 + W)
+        b_cpu = dict(q=torch.randn(2, 4, W, 128, generator=g).bfloat16(),
+                     k=torch.randn(2, 2, L, 128, generator=g).bfloat16(),
+                     v=torch.randn(2, 2, L, 128, generator=g).bfloat16(),
+                     head_w=0.5 + torch.rand(2, 4, generator=g), sens=gen.make_sens(cfg), units=[0, 1])
+    prob = problem_of(cfg, 2)
+    ref = oracle.compress(prob, *(gen.as_numpy(b_cpu[x]) for x in ("q", "k", "v", "head_w", "sens")))
+    out = B.compress(b_cpu["q"].cuda(), b_cpu["k"].cuda(), b_cpu["v"].cuda(), b_cpu["head_w"].cuda(),
+                     b_cpu["sens"].cuda(), params_of(B, prob), want_scores=True)
+    gpu_idx, gpu_bud, gpu_off = (out[x].cpu().numpy() for x in ("indices", "budgets", "offsets"))
+    check_structure(gpu_idx, gpu_bud, gpu_off, prob)
+    check_gather(b_cpu["k"], b_cpu["v"], out["k_out"], out["v_out"], gpu_idx, gpu_off, prob)
+    if Bud >= L:
+        np.testing.assert_array_equal(gen.as_numpy(out["k_out"]).reshape(2, 2, L, 128), gen.as_numpy(b_cpu["k"]))
+        np.testing.assert_array_equal(gen.as_numpy(out["v_out"]).reshape(2, 2, L, 128), gen.as_numpy(b_cpu["v"]))
+    if L > W:
+        gs = out["scores"].double().cpu().numpy()
+        rel = np.abs(gs - ref["scores"]) / np.maximum(np.abs(ref["scores"]), 1e-20)
+        assert rel.max() <= SCORE_RTOL
+        np.testing.assert_array_equal(gpu_idx, oracle.select(prob, gs, gpu_bud, gpu_off))
+
+
+def test_select_exact_ties_and_extremes(B):
+    """Constant and few-valued scores fed straight into ckv_select: the lowest indices win."""
+    Nu, Hkv, L, W = 2, 3, 5000, 32
+    n = L - W
+    rng = np.random.default_rng(5)
+    scores = rng.integers(0, 4, (Nu, Hkv, n)).astype(np.float32)
+    scores[0, 0] = 1.0
+    scores[1, 2, ::7] = -2.5                      # negative values order correctly too
+    budgets = np.array([[42, 4000, 32 + n], [32, 4042, n]], np.int32)   # e = 10 / all / none / ...
+    rows = int(budgets[0].sum())
+    assert budgets[1].sum() == rows
+    offsets = np.concatenate([np.zeros((Nu, 1), np.int32), budgets.cumsum(1).astype(np.int32)], 1)
+    q = torch.zeros(Nu, Hkv, W, 128, dtype=torch.bfloat16, device="cuda")
+    k = torch.zeros(Nu, Hkv, L, 128, dtype=torch.bfloat16, device="cuda")
+    shape = B.make_shape(q, k)
+    assert rows % Hkv == 0
+    P = B.Params(budget_per_head=rows // Hkv, floor_per_head=0)
+    params = B.make_params(P, None, None)
+    ws = B.alloc_workspace(shape, params, "cuda")
+    idx = torch.full((Nu, rows), -1, dtype=torch.int32, device="cuda")
+    B.ckv_select(shape, params, torch.from_numpy(scores).cuda(), torch.from_numpy(budgets).cuda(),
+                 torch.from_numpy(offsets).cuda(), idx, ws)
+    prob = Problem(Nu, Hkv, Hkv, L, W, budget_per_head=rows // Hkv)
+    want = oracle.select(prob, scores.astype(np.float64), budgets, offsets)
+    np.testing.assert_array_equal(idx.cpu().numpy(), want)
+    assert idx[0, :8].tolist() == list(range(8))
+
+
+def test_strided_inputs(B):
+    """K/V living inside a larger allocation (non-dense unit/head/token strides) give the same result."""
+    cfg = gen.shrink(gen.CONFIGS["c2"], n_layers=2, n_q_heads=8, n_kv_heads=2, seq_len=700, budget_per_head=64,
+                     n_needles=4)
+    b = gen.make_batch(cfg, "cuda")
+    prob = problem_of(cfg, 2)
+    P = params_of(B, prob)
+    dense = B.compress(b["q"], b["k"], b["v"], b["head_w"], b["sens"], P, want_scores=True)
+    big_k = torch.zeros(2, 2, 800, 256, dtype=torch.bfloat16, device="cuda")
+    big_v = torch.zeros_like(big_k)
+    big_k[:, :, 50:750, 128:] = b["k"]
+    big_v[:, :, 50:750, 128:] = b["v"]
+    kv, vv = big_k[:, :, 50:750, 128:], big_v[:, :, 50:750, 128:]
+    big_q = torch.zeros(2, 8, 40, 128, dtype=torch.bfloat16, device="cuda")
+    big_q[:, :, 3:35] = b["q"]
+    strided = B.compress(big_q[:, :, 3:35], kv, vv, b["head_w"], b["sens"], P, want_scores=True)
+    for key in ("scores", "indices", "budgets", "k_out", "v_out"):
+        assert torch.equal(dense[key], strided[key]), key
+
+
+def test_compress_host_matches_device_path(B):
+    cfg = gen.shrink(gen.CONFIGS["c2"], n_layers=2, n_q_heads=8, n_kv_heads=2, seq_len=900, budget_per_head=64,
+                     n_needles=4)
+    b = gen.make_batch(cfg, "cpu")
+    prob = problem_of(cfg, 2)
+    P = params_of(B, prob)
+    dev = B.compress(*(b[x].cuda() for x in ("q", "k", "v", "head_w", "sens")), P)
+    shape = B.make_shape(b["q"], b["k"])
+    params = B.make_params(P, b["head_w"], b["sens"])
+    rows = B.rows_per_unit(shape, params)
+    pin = lambda t: t.pin_memory()
+    k_out = pin(torch.zeros(2, rows, 128, dtype=torch.bfloat16))
+    v_out = pin(torch.zeros_like(k_out))
+    idx = pin(torch.zeros(2, rows, dtype=torch.int32))
+    bud = pin(torch.zeros(2, 2, dtype=torch.int32))
+    off = pin(torch.zeros(2, 3, dtype=torch.int32))
+    staging = torch.empty(B.ckv_staging_bytes(shape, params), dtype=torch.uint8, device="cuda")
+    ws = B.alloc_workspace(shape, params, "cuda")
+    B.ckv_compress_host(shape, params, pin(b["q"]), pin(b["k"]), pin(b["v"]), pin(b["head_w"]), pin(b["sens"]),
+                        k_out, v_out, idx, bud, off, staging, ws)
+    assert torch.equal(idx, dev["indices"].cpu()) and torch.equal(bud, dev["budgets"].cpu())
+    assert torch.equal(k_out, dev["k_out"].cpu()) and torch.equal(v_out, dev["v_out"].cpu())
+
+
+def test_deterministic_run_to_run(B):
+    cfg = gen.shrink(gen.CONFIGS["c2"], n_layers=2, seq_len=3000, budget_per_head=128, n_needles=8)
+    b = gen.make_batch(cfg, "cuda")
+    P = params_of(B, problem_of(cfg, 2))
+    a = B.compress(b["q"], b["k"], b["v"], b["head_w"], b["sens"], P, want_scores=True)
+    c = B.compress(b["q"], b["k"], b["v"], b["head_w"], b["sens"], P, want_scores=True)
+    for key in ("scores", "indices", "budgets", "k_out", "v_out", "entropy"):
+        assert torch.equal(a[key], c[key]), key

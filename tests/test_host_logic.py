@@ -1,0 +1,157 @@
+"""CPU-only checks of the library's host side: the shared object loads and exports the whole C ABI,
+argument errors are reported before anything is launched, the integer budget split used by the
+device code agrees with the oracle and with brute force, and the multi-rank sharding works under
+gloo with two processes."""
+import ctypes as C
+import os
+import re
+import subprocess
+import sys
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2602_08686_b200 import binding as B
+from paper_2602_08686_b200 import build as ckv_build
+from paper_2602_08686_b200.sharding import shard_units
+from test_oracle_pins import brute_allocate
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    ckv_build.build_lib()
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "ckv.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    names = sorted(set(re.findall(r"\b(ckv_[a-z_]+)\s*\(", header)))
+    assert {"ckv_score", "ckv_budget", "ckv_select", "ckv_gather", "ckv_compress"} <= set(names)
+    lib = B.lib()
+    for n in names:
+        assert hasattr(lib, n), n
+    assert B.ckv_version() >= 100
+    assert B.status_string(B.ERR_TIMEOUT)
+
+
+def llama_shape(L=32768, W=32, Nu=2, H=32, Hkv=8, d=128, dtype=B.BF16):
+    return B.ckv_shape(Nu, H, Hkv, d, L, W, dtype, 0, H * W * d, W * d, d, Hkv * L * d, L * d, d)
+
+
+def default_params(**kw):
+    base = dict(pool_kind=B.POOL_MAX, pool_size=7, budget_per_head=512, floor_per_head=1, n_buckets=16,
+                bucket_override=-1, head_w_stride_unit=32, sens_stride_unit=0)
+    base.update(kw)
+    return B.ckv_params(*[base[k] for k in ("pool_kind", "pool_size", "budget_per_head", "floor_per_head",
+                                            "n_buckets", "bucket_override", "head_w_stride_unit",
+                                            "sens_stride_unit")])
+
+
+def test_argument_errors_are_found_on_the_host():
+    lib = B.lib()
+    s, p = llama_shape(), default_params()
+    assert B.ckv_workspace_bytes(s, p) > 0
+    fake = C.c_void_p(256 * 1024)      # never dereferenced: every call below fails validation first
+    big = 1 << 40
+
+    def score(shape, params, ws=fake, ws_bytes=big, q=fake):
+        return lib.ckv_score(C.byref(shape), C.byref(params), q, fake, fake, fake, fake, ws, ws_bytes, None)
+
+    assert score(llama_shape(d=64), p) == B.ERR_UNSUPPORTED
+    assert score(llama_shape(W=65), p) == B.ERR_UNSUPPORTED
+    assert score(llama_shape(H=30), p) == B.ERR_INVALID_ARG
+    assert score(llama_shape(L=16), p) == B.ERR_INVALID_ARG                       # window > seq_len
+    assert score(s, default_params(pool_size=4)) == B.ERR_INVALID_ARG
+    assert score(s, default_params(pool_size=17)) == B.ERR_INVALID_ARG
+    assert score(s, default_params(budget_per_head=16)) == B.ERR_INVALID_ARG      # B < W
+    assert score(s, default_params(floor_per_head=500)) == B.ERR_INVALID_ARG      # f > B - W
+    assert score(s, default_params(bucket_override=16)) == B.ERR_INVALID_ARG
+    assert score(s, p, q=None) == B.ERR_INVALID_ARG
+    assert score(s, p, q=C.c_void_p(256 * 1024 + 2)) == B.ERR_INVALID_ARG         # misaligned
+    assert score(s, p, ws=None) == B.ERR_WORKSPACE
+    assert score(s, p, ws_bytes=1024) == B.ERR_WORKSPACE
+    bad = llama_shape()
+    bad.kv_stride_tok = 130                                                       # rows not 16-byte aligned
+    assert score(bad, p) == B.ERR_INVALID_ARG
+    assert B.ckv_workspace_bytes(llama_shape(d=64), p) == 0
+    assert lib.ckv_gather(C.byref(s), C.byref(p), None, fake, fake, fake, fake, fake, None) == B.ERR_INVALID_ARG
+    assert lib.ckv_compress_host(C.byref(s), C.byref(p), fake, fake, fake, fake, fake, fake, fake, fake, fake, fake,
+                                 fake, 16, fake, big, None) == B.ERR_WORKSPACE    # staging too small
+
+
+def test_workspace_grows_with_the_problem():
+    p = default_params()
+    a = B.ckv_workspace_bytes(llama_shape(L=4096), p)
+    b = B.ckv_workspace_bytes(llama_shape(L=32768), p)
+    c = B.ckv_workspace_bytes(llama_shape(L=32768, Nu=4), p)
+    assert 0 < a < b < c
+    assert B.ckv_staging_bytes(llama_shape(L=4096), p) > 2 * 2 * 8 * 4096 * 128 * 2
+
+
+def test_budget_split_matches_oracle_and_brute_force():
+    rng = np.random.default_rng(11)
+    for Hkv in (1, 2, 3, 4, 8):
+        for _ in range(300):
+            n = int(rng.integers(1, 60))
+            f = int(rng.integers(0, n + 1))
+            P = int(rng.integers(f * Hkv, n * Hkv + 1))
+            lo = max(f, 1)
+            dem = rng.integers(lo, max(lo, n) + 1, Hkv)
+            if rng.random() < 0.4:
+                dem[:] = dem[0]                                                   # equal demands
+            got = B.ckv_allocate_rows_host(n, f, P, dem)
+            assert got == list(oracle.allocate(n, f, P, dem)), (n, f, P, dem)
+            if Hkv <= 4:
+                assert got == brute_allocate(n, f, P, dem)
+    # sizes of the real workloads
+    for n, f, B_, Hkv in ((32736, 1, 512, 8), (131040, 1, 2048, 8), (65472, 8, 128, 4)):
+        for _ in range(50):
+            dem = rng.integers(max(f, 1), n + 1, Hkv) // rng.integers(1, 2000, Hkv) + max(f, 1)
+            dem = np.minimum(dem, n)
+            P = Hkv * (B_ - (64 if Hkv == 4 else 32))
+            got = B.ckv_allocate_rows_host(n, f, P, dem)
+            assert got == list(oracle.allocate(n, f, P, dem))
+            assert sum(got) == P and min(got) >= f and max(got) <= n
+
+
+def test_shard_units_partitions():
+    for n in (1, 7, 32, 512):
+        for world in (1, 2, 3, 8):
+            parts = [shard_units(n, r, world) for r in range(world)]
+            assert sorted(x for p in parts for x in p) == list(range(n))
+            sizes = [len(p) for p in parts]
+            assert max(sizes) - min(sizes) <= 1
+
+
+_GLOO_WORKER = r"""
+import os, sys, torch, torch.distributed as dist
+sys.path.insert(0, sys.argv[1])
+from paper_2602_08686_b200.sharding import shard_units, max_over_ranks
+dist.init_process_group("gloo", init_method="tcp://127.0.0.1:" + sys.argv[2], rank=int(sys.argv[3]), world_size=2)
+rank = dist.get_rank()
+mine = shard_units(33, rank, 2)
+t = torch.zeros(33, dtype=torch.int64); t[list(mine)] = 1
+dist.all_reduce(t)
+assert (t == 1).all(), t
+elapsed = max_over_ranks(1.0 + rank)
+assert elapsed == 2.0, elapsed
+total = torch.tensor([float(len(mine))]); dist.all_reduce(total)
+assert total.item() == 33.0
+dist.barrier(); dist.destroy_process_group()
+print("rank", rank, "ok")
+"""
+
+
+def test_two_rank_sharding_under_gloo(tmp_path):
+    """World size 2 on CPU: the ranks' shards cover every unit once and the timing reduction is a MAX."""
+    script = tmp_path / "worker.py"
+    script.write_text(_GLOO_WORKER)
+    port = str(29000 + os.getpid() % 2000)
+    procs = [subprocess.Popen([sys.executable, str(script), ROOT, port, str(r)], stdout=subprocess.PIPE,
+                              stderr=subprocess.STDOUT) for r in range(2)]
+    outs = [p.communicate(timeout=180)[0].decode() for p in procs]
+    for p, o in zip(procs, outs):
+        assert p.returncode == 0, o
