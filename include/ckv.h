@@ -156,6 +156,12 @@ ckv_status ckv_compress_host(const ckv_shape* shape, const ckv_params* params, c
  * CKV_ERR_TIMEOUT), or CKV_ERR_CUDA if the stream is in error. */
 ckv_status ckv_device_status(const void* ws, void* stream);
 
+/* Diagnostic switch for the window-score scan: 0 = automatic (tensor-core kernel for bf16 inputs with
+ * window 16, 32 or 64 and L >= 128, plain kernels otherwise), 1 = always the plain kernels, 2 = require
+ * the tensor-core kernel (ckv_score returns CKV_ERR_UNSUPPORTED where it does not apply).  Process-wide;
+ * returns the previous setting, or -1 for an invalid value. */
+int ckv_set_score_path(int path);
+
 /* Number of kernel launches this process has queued through the library so far. */
 int64_t ckv_kernel_launches(void);
 

@@ -82,6 +82,11 @@ def ckv_version() -> int:
     return lib().ckv_version()
 
 
+def ckv_set_score_path(path: int) -> int:
+    """0 automatic, 1 plain kernels, 2 tensor-core kernel required; returns the previous setting."""
+    return int(lib().ckv_set_score_path(int(path)))
+
+
 def ckv_kernel_launches() -> int:
     return int(lib().ckv_kernel_launches())
 

@@ -7,6 +7,7 @@
 namespace ckv {
 
 static std::atomic<int64_t> g_launches{0};
+static std::atomic<int> g_score_path{0};  // 0 = automatic, 1 = plain kernels, 2 = tensor-core kernel
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
 static size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
@@ -25,6 +26,12 @@ WsLayout ws_layout(const ckv_shape& s, const ckv_params&) {
   w.scores = o, o = align_up(o + Nu * Hkv * (n ? n : 1) * sizeof(float));
   w.bucket = o, o = align_up(o + Nu * sizeof(int32_t));
   w.entropy = o, o = align_up(o + Nu * sizeof(float));
+  if (s.dtype == CKV_BF16) {
+    const TcLayout t = tc_layout(s);
+    w.tc_part = o, o = align_up(o + t.part_bytes);
+    w.tc_stat = o, o = align_up(o + t.stat_bytes);
+    w.tc_flags = o, o = align_up(o + t.flag_bytes);
+  }
   w.total = o;
   return w;
 }
@@ -95,8 +102,16 @@ static ckv_status score_impl(const ckv_shape& s, const ckv_params& p, const void
   const WsLayout w = ws_layout(s, p);
   CKV_CUDA(cudaMemsetAsync(ws + w.status, 0, 256, st));
   float* csum = reinterpret_cast<float*>(ws + w.csum);
-  CKV_CUDA(launch_score_plain(s, q, k, csum, reinterpret_cast<float2*>(ws + w.part),
-                              reinterpret_cast<float2*>(ws + w.stat), w.nblk, st));
+  const int path = g_score_path.load(std::memory_order_relaxed);
+  const bool tc_ok = score_tc_supported(s) && s.seq_len >= 128;
+  if (path == 2 && !tc_ok) return CKV_ERR_UNSUPPORTED;
+  if (tc_ok && path != 1) {
+    CKV_CUDA(launch_score_tc(s, q, k, csum, ws + w.tc_part, ws + w.tc_stat, reinterpret_cast<int*>(ws + w.tc_flags),
+                             reinterpret_cast<int*>(ws + w.status), st));
+  } else {
+    CKV_CUDA(launch_score_plain(s, q, k, csum, reinterpret_cast<float2*>(ws + w.part),
+                                reinterpret_cast<float2*>(ws + w.stat), w.nblk, st));
+  }
   CKV_CUDA(launch_epilogue(s, p, csum, head_w, scores, colmass, st));
   return CKV_OK;
 }
@@ -266,6 +281,11 @@ ckv_status ckv_device_status(const void* ws, void* stream) {
     return CKV_ERR_CUDA;
   if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return CKV_ERR_CUDA;
   return word == 0 ? CKV_OK : CKV_ERR_TIMEOUT;
+}
+
+int ckv_set_score_path(int path) {
+  if (path < 0 || path > 2) return -1;
+  return g_score_path.exchange(path, std::memory_order_relaxed);
 }
 
 int64_t ckv_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }

@@ -34,6 +34,15 @@ def B():
     return binding
 
 
+@pytest.fixture(params=["auto", "plain"])
+def score_path(request, B):
+    """Runs a case once with the automatic choice (tensor-core scan where it applies) and once with the
+    plain kernels forced."""
+    prev = B.ckv_set_score_path(1 if request.param == "plain" else 0)
+    yield request.param
+    B.ckv_set_score_path(prev)
+
+
 def problem_of(cfg, Nu, **kw):
     prob = Problem(Nu, cfg.n_q_heads, cfg.n_kv_heads, cfg.seq_len, cfg.window, head_dim=cfg.head_dim,
                    dtype=oracle.BF16 if cfg.dtype == "bf16" else oracle.F32, pool_kind=cfg.pool_kind,
@@ -204,21 +213,47 @@ def test_config1_fp32_whole(B):
     run_case(B, gen.CONFIGS["c1"])
 
 
-@pytest.mark.parametrize("L", [4096, 4000, 1111])
-def test_llama_shape_small(B, L):
+@pytest.mark.parametrize("L", [4096, 4000, 1111, 128, 129])
+def test_llama_shape_small(B, L, score_path):
     """Config 2's head layout at lengths that span several key tiles and leave a ragged tail."""
-    cfg = gen.shrink(gen.CONFIGS["c2"], n_layers=2, seq_len=L, budget_per_head=128, n_needles=8)
+    cfg = gen.shrink(gen.CONFIGS["c2"], n_layers=2, seq_len=L, budget_per_head=min(128, L // 2),
+                     n_needles=8 if L > 1000 else 2)
     run_case(B, cfg)
 
 
-def test_heavy_tail_keys(B):
+def test_tensor_core_path_is_taken_and_agrees_with_plain(B):
+    """bf16, W 32, L >= 128 must run the tcgen05 kernel (path 2 = required) and match the plain kernels."""
+    cfg = gen.shrink(gen.CONFIGS["c2"], n_layers=3, seq_len=5000, budget_per_head=128, n_needles=8)
+    b = gen.make_batch(cfg, "cuda")
+    P = params_of(B, problem_of(cfg, 3))
+    prev = B.ckv_set_score_path(2)
+    try:
+        tc = B.compress(b["q"], b["k"], b["v"], b["head_w"], b["sens"], P, want_scores=True)
+        assert B.ckv_device_status(tc["ws"]) == B.OK
+        B.ckv_set_score_path(1)
+        pl = B.compress(b["q"], b["k"], b["v"], b["head_w"], b["sens"], P, want_scores=True)
+    finally:
+        B.ckv_set_score_path(prev)
+    rel = ((tc["scores"] - pl["scores"]).abs() / pl["scores"].abs().clamp_min(1e-20)).max().item()
+    assert rel < 1e-4, rel
+
+
+@pytest.mark.parametrize("G,W", [(1, 32), (2, 64), (3, 16), (9, 16), (5, 32)])
+def test_group_sizes_and_windows(B, G, W):
+    """Row blocks: G*W below, equal to and above 128 rows (several blocks, the last one partial)."""
+    cfg = gen.shrink(gen.CONFIGS["c2"], n_layers=2, n_q_heads=2 * G, n_kv_heads=2, seq_len=1500, window=W,
+                     budget_per_head=100, n_needles=4)
+    run_case(B, cfg)
+
+
+def test_heavy_tail_keys(B, score_path):
     """Config 4's structure (Student-t key scales, stratified needles) at a length the oracle finishes."""
     cfg = gen.shrink(gen.CONFIGS["c4"], n_layers=2, seq_len=8192, budget_per_head=128, n_needles=16)
     run_case(B, cfg)
 
 
 @pytest.mark.parametrize("budget", [128, 512])
-def test_qwen_shape_L4096(B, budget):
+def test_qwen_shape_L4096(B, budget, score_path):
     """Config 5 at L 4096: GQA 7, W 64, AVG pool 5, floor 8, one low-reliability group per layer."""
     cfg = gen.shrink(gen.c5_point(4096, budget), n_layers=2, batch=2)
     run_case(B, cfg)
