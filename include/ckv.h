@@ -152,6 +152,34 @@ ckv_status ckv_compress_host(const ckv_shape* shape, const ckv_params* params, c
                              int32_t* indices_host, int32_t* budgets_host, int32_t* offsets_host,
                              void* staging, size_t staging_bytes, void* ws, size_t ws_bytes, void* stream);
 
+/*
+ * ckv_score without a work-space argument, for callers that cannot allocate device memory: code
+ * that runs inside another framework's memory plan or under a fixed memory budget, where every
+ * byte of HBM was handed out before this library is called and cudaMalloc (or a framework
+ * allocator that may fall back to it) is off limits, or too slow, at that point.  The paper has
+ * no counterpart to this entry point; it computes exactly what ckv_score computes, with the same
+ * kernels, and differs only in where the intermediate data lives.
+ *
+ * The scratch is a fixed array of CKV_NOALLOC_SCRATCH_BYTES bytes in the library's own device
+ * image: every GPU on which the library is loaded holds it from load until the process exits.
+ * Problems whose ckv_workspace_bytes() exceeds that size are refused with CKV_ERR_WORKSPACE before
+ * anything is launched (use ckv_score with a caller-owned work space for those).
+ *   - Nothing is allocated or freed, by the CUDA runtime or otherwise.  The first call on a device
+ *     looks up the array's device address (one runtime query, remembered per device); make that
+ *     first call outside any stream capture.
+ *   - All calls on one device share the array and it keeps whatever the last call left in it; the
+ *     entry point clears the few words that must start at zero.  Two calls whose kernels can run at
+ *     the same time on one device (different streams without an ordering between them) race on it:
+ *     serialise them.
+ *   - The device status word lives inside the array, so ckv_device_status() cannot report on this
+ *     variant.
+ * Arguments, layouts, outputs and the remaining error codes are those of ckv_score.
+ */
+#define CKV_NOALLOC_SCRATCH_BYTES (16u << 20)
+ckv_status ckv_score_noalloc(const ckv_shape* shape, const ckv_params* params, const void* q_win,
+                             const void* k, const float* head_w, float* scores, float* colmass,
+                             void* stream);
+
 /* Synchronises `stream` and returns the status word device code wrote into `ws` (CKV_OK or
  * CKV_ERR_TIMEOUT), or CKV_ERR_CUDA if the stream is in error. */
 ckv_status ckv_device_status(const void* ws, void* stream);

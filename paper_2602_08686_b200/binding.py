@@ -57,6 +57,7 @@ def lib() -> C.CDLL:
         L.ckv_staging_bytes.restype = sz
         L.ckv_staging_bytes.argtypes = [shp, prm]
         L.ckv_score.argtypes = [shp, prm, vp, vp, fp, fp, fp, vp, sz, vp]
+        L.ckv_score_noalloc.argtypes = [shp, prm, vp, vp, fp, fp, fp, vp]
         L.ckv_budget.argtypes = [shp, prm, fp, fp, fp, i32p, i32p, i32p, fp, vp, sz, vp]
         L.ckv_select.argtypes = [shp, prm, fp, i32p, i32p, i32p, vp, sz, vp]
         L.ckv_gather.argtypes = [shp, prm, vp, vp, i32p, i32p, vp, vp, vp]
@@ -67,7 +68,7 @@ def lib() -> C.CDLL:
         L.ckv_status_string.restype = C.c_char_p
         L.ckv_status_string.argtypes = [C.c_int]
         L.ckv_allocate_rows_host.argtypes = [C.c_int, C.c_int64, C.c_int64, C.c_int64, vp, vp]
-        for name in ("ckv_score", "ckv_budget", "ckv_select", "ckv_gather", "ckv_compress", "ckv_compress_host",
+        for name in ("ckv_score", "ckv_score_noalloc", "ckv_budget", "ckv_select", "ckv_gather", "ckv_compress", "ckv_compress_host",
                      "ckv_device_status", "ckv_version", "ckv_allocate_rows_host"):
             getattr(L, name).restype = C.c_int
         _lib = L
@@ -162,6 +163,16 @@ def rows_per_unit(shape: ckv_shape, params: ckv_params) -> int:
 def ckv_score(shape, params, q_win, k, head_w, scores, colmass, ws, stream=None):
     _check(lib().ckv_score(C.byref(shape), C.byref(params), _ptr(q_win), _ptr(k), _ptr(head_w), _ptr(scores),
                            _ptr(colmass), _ptr(ws), ws.numel(), _stream(stream)), "ckv_score")
+
+
+NOALLOC_SCRATCH_BYTES = 16 << 20
+
+
+def ckv_score_noalloc(shape, params, q_win, k, head_w, scores, colmass, stream=None):
+    """ckv_score on the library's own fixed scratch (no work space, nothing allocated); problems that need
+    more than NOALLOC_SCRATCH_BYTES raise CkvError with ERR_WORKSPACE.  Calls on one device must not overlap."""
+    _check(lib().ckv_score_noalloc(C.byref(shape), C.byref(params), _ptr(q_win), _ptr(k), _ptr(head_w),
+                                   _ptr(scores), _ptr(colmass), _stream(stream)), "ckv_score_noalloc")
 
 
 def ckv_budget(shape, params, scores, colmass, sens, budgets, offsets, bucket, entropy, ws, stream=None):

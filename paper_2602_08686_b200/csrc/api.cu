@@ -1,6 +1,7 @@
 // Host side of the C ABI: argument validation, work-space layout and the launch sequences.
 #include <atomic>
 #include <cstring>
+#include <mutex>
 
 #include "ckv_common.cuh"
 
@@ -315,4 +316,47 @@ int ckv_allocate_rows_host(int hkv, int64_t n, int64_t f, int64_t P, const int64
 }
 
 }  // extern "C"
+#pragma GCC visibility pop
+
+// ---------------------------------------------------------------------------------------------
+// Scratch for ckv_score_noalloc: a fixed array in every device's global memory, present from the
+// moment the library is loaded on that device until the process exits.  Host code must never hand
+// the symbol itself to a kernel (on the host the name is only a stand-in); it asks the runtime for
+// the device address once per device and passes that.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[CKV_NOALLOC_SCRATCH_BYTES];
+
+namespace ckv {
+constexpr int kMaxDevices = 64;
+static std::mutex g_noalloc_mutex;
+static void* g_noalloc_ptr[kMaxDevices] = {};
+
+// Device address of the fixed scratch on the current device (looked up on first use per device).
+static ckv_status noalloc_scratch(char** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return CKV_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+  if (!g_noalloc_ptr[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return CKV_ERR_CUDA;
+    g_noalloc_ptr[dev] = p;
+  }
+  *out = static_cast<char*>(g_noalloc_ptr[dev]);
+  return CKV_OK;
+}
+}  // namespace ckv
+
+#pragma GCC visibility push(default)
+extern "C" ckv_status ckv_score_noalloc(const ckv_shape* shape, const ckv_params* params, const void* q_win,
+                                        const void* k, const float* head_w, float* scores, float* colmass,
+                                        void* stream) {
+  CKV_TRY(check_shape(shape));
+  CKV_TRY(check_params(shape, params));
+  if (!all_aligned16({q_win, k}) || !all_aligned4({head_w, scores, colmass})) return CKV_ERR_INVALID_ARG;
+  if (ws_layout(*shape, *params).total > (size_t)CKV_NOALLOC_SCRATCH_BYTES) return CKV_ERR_WORKSPACE;
+  char* scratch = nullptr;
+  CKV_TRY(noalloc_scratch(&scratch));
+  // score_impl zeroes the status word and the scan's counters before its kernels read them; the rest
+  // of the scratch is written before it is read, so what the previous call left behind is harmless.
+  return score_impl(*shape, *params, q_win, k, head_w, scores, colmass, scratch, (cudaStream_t)stream);
+}
 #pragma GCC visibility pop
