@@ -64,6 +64,8 @@ def lib() -> C.CDLL:
         L.ckv_compress.argtypes = [shp, prm, vp, vp, vp, fp, fp, vp, vp, i32p, i32p, i32p, fp, i32p, fp, vp, sz, vp]
         L.ckv_compress_host.argtypes = [shp, prm, vp, vp, vp, fp, fp, vp, vp, i32p, i32p, i32p, vp, sz, vp, sz, vp]
         L.ckv_device_status.argtypes = [vp, vp]
+        L.ckv_set_tunable.argtypes = [C.c_char_p, C.c_int]
+        L.ckv_set_tunable.restype = C.c_int
         L.ckv_kernel_launches.restype = C.c_int64
         L.ckv_status_string.restype = C.c_char_p
         L.ckv_status_string.argtypes = [C.c_int]
@@ -86,6 +88,14 @@ def ckv_version() -> int:
 def ckv_set_score_path(path: int) -> int:
     """0 automatic, 1 plain kernels, 2 tensor-core kernel required; returns the previous setting."""
     return int(lib().ckv_set_score_path(int(path)))
+
+
+def ckv_set_tunable(name: str, value: int) -> int:
+    """Schedule knob of the tensor-core scan ("run_tiles", "lag_slack_pct", "l2_hints"); returns the previous value."""
+    prev = int(lib().ckv_set_tunable(name.encode(), int(value)))
+    if prev < 0:
+        raise ValueError(f"unknown tunable or value out of range: {name}={value}")
+    return prev
 
 
 def ckv_kernel_launches() -> int:

@@ -289,6 +289,11 @@ int ckv_set_score_path(int path) {
   return g_score_path.exchange(path, std::memory_order_relaxed);
 }
 
+int ckv_set_tunable(const char* name, int value) {
+  if (!name) return -1;
+  return set_tc_tunable(name, value);
+}
+
 int64_t ckv_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
 
 const char* ckv_status_string(ckv_status status) {

@@ -25,7 +25,7 @@ struct WsLayout {
   size_t scores;   // float [Nu, Hkv, n]      likewise
   size_t bucket;   // int32 [Nu]
   size_t entropy;  // float [Nu]
-  size_t tc_part;  // float2 [C, 2*RPC, 128]   partial row statistics of the tensor-core scan
+  size_t tc_part;  // float2 [C, T+2, 128]     partial row statistics of the tensor-core scan
   size_t tc_stat;  // float2 [C, 128]          final row statistics per chunk
   size_t tc_flags; // int32 [C, 5]             completion counters and ready flags
   size_t total;
@@ -34,12 +34,13 @@ struct WsLayout {
 
 // Sizes of the tensor-core scan's scratch for a shape (chunks of 128 query rows x whole key range).
 struct TcLayout {
-  int RB, T, RPC;
+  int RB, T;
   int64_t C;
   size_t part_bytes, stat_bytes, flag_bytes;
 };
 TcLayout tc_layout(const ckv_shape& s);
 bool score_tc_supported(const ckv_shape& s);
+int set_tc_tunable(const char* name, int value);
 cudaError_t launch_score_tc(const ckv_shape& s, const void* q, const void* k, float* csum, void* part, void* stat,
                             int* flags, int* status, cudaStream_t st);
 

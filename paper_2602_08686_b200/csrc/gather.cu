@@ -24,6 +24,11 @@ __global__ void __launch_bounds__(256) gather_kernel(ckv_shape s, int rows_per_h
     int g = 0;
     while (g + 1 < Hkv && r >= off[g + 1]) ++g;
     const int t = indices[row];
+    if ((unsigned)t >= (unsigned)s.seq_len) {  // never produced by ckv_select; guards against foreign index buffers
+      k_out[i] = make_uint4(0u, 0u, 0u, 0u);
+      v_out[i] = make_uint4(0u, 0u, 0u, 0u);
+      continue;
+    }
     const int64_t src =
         ((int64_t)u * s.kv_stride_unit + (int64_t)g * s.kv_stride_head + (int64_t)t * s.kv_stride_tok) / elems_per_vec +
         piece;

@@ -7,16 +7,31 @@
 //        merges them in a fixed order into (max, max + log2 sum).
 //   P2 (column sums)     D[key, row]  = K_tile . Q_blk^T   (the same shared-memory tiles, operands
 //        swapped): one TMEM lane per key, so c_h[t] = sum_i 2^(x[i,t] - bias_i) is thread-local.
-// A "chunk" is one (unit, KV head, block of 128 query rows); a "run" is up to four consecutive key
-// tiles of a chunk.  CTA b handles P1 runs b, b+grid, ... and, interleaved, the P2 runs that trail
-// them by a fixed lag, so the second read of a K tile comes from L2 while its chunk's statistics are
-// long complete.  K and Q tiles arrive by TMA (128-byte swizzle) and feed tcgen05.mma directly; the
-// accumulators live in TMEM (four 128-column buffers) and are read back with tcgen05.ld.
+// A "chunk" is one (unit, KV head, block of 128 query rows); a "run" is a few consecutive key tiles of
+// a chunk.  CTA b takes P1 runs b, b+grid, ... and the P2 runs that trail them by a fixed lag, one tile
+// of each in turn, so the second read of a K tile comes from L2 while its chunk's statistics are
+// complete.  Warp roles:
+//   warp 0       producer (one thread): computes the schedule, issues the TMA loads and hands every
+//                sub-item (one tile of one pass) to the others through a descriptor ring in shared
+//                memory.  Sub-item j uses K stage j % 5 and TMEM buffer j % 4.  P1 tiles sit at even j,
+//                P2 tiles at odd j (a slot without work carries a no-op), and once P1 has ended P2
+//                takes both.  A P2 chunk whose statistics are not final yet never blocks P1: its slot
+//                carries a no-op and the tile is issued later.
+//   warps 1, 19  MMA issuers (one thread each, even / odd j): tcgen05.mma M = N = K = 128 into one of four
+//                128-column TMEM buffers.
+//   warps 2..17  consumers: four groups, one per TMEM buffer, each with one warp per lane quadrant,
+//                read the accumulators back with tcgen05.ld.  Groups 0 and 2 see the P1 tiles.
+//   warp 18      scout: walks the CTA's P2 runs ahead of the producer, waits for a chunk's statistics
+//                and stages its 128 row biases in shared memory.
+// K and Q tiles arrive by TMA (128-byte swizzle) and feed tcgen05.mma directly.
 //
-// Every wait is bounded: an mbarrier or flag wait that exceeds its time limit records
-// CKV_ERR_TIMEOUT in the work space's status word and the CTA winds down (frees TMEM, returns).
+// Every wait is bounded: an mbarrier or flag wait that exceeds its time limit records a code in the
+// work space's status word (reported as CKV_ERR_TIMEOUT) and the CTA winds down (frees TMEM, returns).
 #include <cuda.h>
 #include <cuda_bf16.h>
+
+#include <atomic>
+#include <string>
 
 #include "ckv_common.cuh"
 
@@ -24,15 +39,20 @@ namespace ckv {
 namespace {
 
 constexpr int kTile = 128;        // keys per tile, also query rows per block
-constexpr int kStages = 4;        // K-tile ring
-constexpr int kTmemBufs = 4;      // accumulator buffers of 128 columns
-constexpr int kRun = 4;           // key tiles per run
-constexpr int kBiasSlots = 8;     // >= kStages + kTmemBufs
-constexpr int kConsumerWarps = 8; // two sets of four (one warp per TMEM lane quadrant)
-constexpr int kThreads = 32 * (2 + kConsumerWarps);
+constexpr int kStages = 5;        // K-tile ring
+constexpr int kFullBars = 2 * kStages;
+constexpr int kTmemBufs = 4;      // accumulator buffers of 128 columns, one per consumer group
+constexpr int kRing = 16;         // descriptor slots
+static_assert(kRing >= kStages + kTmemBufs, "a descriptor slot is reused only after its readers are done");
+constexpr int kBiasBufs = 4;      // bias vectors of the most recent P2 chunks
+constexpr int kConsumerWarps = 16;
+constexpr int kScoutWarp = 2 + kConsumerWarps;
+constexpr int kMma2Warp = 3 + kConsumerWarps;
+constexpr int kThreads = 32 * (4 + kConsumerWarps);
 constexpr uint32_t kHalfBytes = 128 * 128;          // 128 rows x 64 bf16
 constexpr uint32_t kTileBytes = 2 * kHalfBytes;     // 128 rows x 128 bf16
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+constexpr float kMinRowMax = -1.0e30f;              // stands in for "no visible key yet"
 
 // x = (q.k) * log2(e) / sqrt(128)
 constexpr float kScale = 0.12751743074602467f;
@@ -40,53 +60,48 @@ constexpr float kScale = 0.12751743074602467f;
 // UMMA instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = 128.
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 
+// Tunables of the schedule (process-wide; see ckv_set_tunable).
+std::atomic<int> g_run_tiles{4};        // key tiles per run
+std::atomic<int> g_lag_slack_pct{200};  // extra lag of the P2 stream, in percent of the grid size
+std::atomic<int> g_l2_hints{1};         // 1: P1 loads keep their lines (evict_last), P2 loads release them
+
 struct TcArgs {
   int Nu, H, Hkv, G, L, W, n;
   int RB, hpb;          // row blocks per KV group; query heads per row block (128 / W)
-  int T, RPC, C;        // key tiles per chunk; runs per chunk; chunks
+  int T, run, RPC, C;   // key tiles per chunk; tiles per run; runs per chunk; chunks
   int NR, DR;           // runs in total; lag of the P2 stream behind the P1 stream, in runs
-  int expected;         // partial flushes per (chunk, lane quadrant)
-  uint32_t q_half_bytes;
+  int ppr, expected;    // partial pairs per run (1 or 2); pairs per (chunk, lane quadrant)
+  int hints;
+  uint32_t q_bytes;     // bytes of one Q block load
+  int q_split;          // the Q box holds fewer than 128 rows: its two halves are loaded separately
   float* csum;
-  float2* part;         // [C][2*RPC][128]
-  float2* stat;         // [C][128]
+  float2* part;         // [C][ppr*RPC][128] partial (row max, row sum) per run and consumer group
+  float2* stat;         // [C][128]          (row max, row max + log2 row sum)
   int* done;            // [C][4]
   int* ready;           // [C]
   int* status;
 };
 
-struct SubItem {
-  int type;  // 0 = P1, 1 = P2
-  int chunk, tile, k, tr, run_in_chunk;
-};
+// Optional event trace of one CTA (a profiling build defines CKV_TC_TRACE).
+#ifdef CKV_TC_TRACE
+__device__ long long g_tc_trace[6][1024];
+#define TC_TRACE(ev, jj) \
+  do { if (blockIdx.x == 5 && (jj) < 1024) g_tc_trace[ev][jj] = clock64(); } while (0)
+#else
+#define TC_TRACE(ev, jj) do {} while (0)
+#endif
 
-// The fixed sequence of sub-items of one CTA; every warp role walks it independently.
-struct Sched {
-  int b, grid, m, phase, k;
-  __device__ Sched(int b_, int grid_) : b(b_), grid(grid_), m(0), phase(0), k(0) {}
-  __device__ bool next(const TcArgs& a, SubItem& s) {
-    while (true) {
-      const int rho1 = b + m * grid;
-      if (phase == 0 && rho1 - a.DR >= a.NR) return false;
-      const int rho = phase == 0 ? rho1 : rho1 - a.DR;
-      if (rho >= 0 && rho < a.NR) {
-        const int chunk = rho / a.RPC, ric = rho - chunk * a.RPC;
-        const int tr = min(kRun, a.T - ric * kRun);
-        if (k < tr) {
-          s.type = phase, s.chunk = chunk, s.run_in_chunk = ric, s.tr = tr, s.k = k, s.tile = ric * kRun + k;
-          ++k;
-          return true;
-        }
-      }
-      k = 0;
-      if (phase == 0) {
-        phase = 1;
-      } else {
-        phase = 0;
-        ++m;
-      }
-    }
-  }
+// What the producer tells the other warps about sub-item j (ring slot j % kRing).
+enum : int { kP1 = 0, kP2 = 1, kNop = 2, kStop = 3 };
+struct __align__(16) Desc {
+  int type;       // kP1, kP2, kNop, kStop; bit 9: phase parity of the stream's q_full barrier to wait for
+  int chunk;
+  int tile;       // key tile within the chunk
+  int part_slot;  // P1: where this group's pair of the run goes, or -1 while the run goes on
+  int first;      // P1: this group's first tile of the run (reset the running pair)
+  int head0;      // P2: index (u * H + head) of the first query head of the row block
+  int n_heads;    // P2: query heads of the row block that exist
+  int nbias_buf;  // P2: which bias vector belongs to the tile's chunk
 };
 
 // ------------------------------------------------------------------------------------ PTX helpers
@@ -126,7 +141,10 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volat
   for (int it = 0;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 255) == 255) {
-      if (*abort_flag) return false;
+      if (*abort_flag) {
+        atomicCAS(status + 1 + (code & 7), 0, code);  // which wait each role was in when the CTA gave up
+        return false;
+      }
       if (global_ns() - t0 > kWaitLimitNs) {
         *abort_flag = 1;
         atomicCAS(status, 0, code);
@@ -142,27 +160,42 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   return mbar_wait_slow(bar, parity, abort_flag, status, code);
 }
 
-__device__ __forceinline__ void tma_load_4d(const CUtensorMap* map, uint32_t dst, uint32_t bar, int c0, int c1, int c2,
-                                            int c3) {
+__device__ __forceinline__ void tma_load_5d(const CUtensorMap* map, uint32_t dst, uint32_t bar, int c0, int c1, int c2,
+                                            int c3, int c4, uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%3, %4, %5, %6, %7}], [%2], %8;"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4),
+      "l"(policy)
       : "memory");
+}
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t policy_evict_normal() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
+  return p;
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows 128 bytes apart, groups of
-// eight rows 1024 bytes apart.
-__device__ __forceinline__ uint64_t umma_desc(uint32_t addr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((addr >> 4) & 0x3fff);
-  d |= (uint64_t)1 << 16;               // leading byte offset (unused for swizzled K-major), canonical value 1
-  d |= (uint64_t)(1024 >> 4) << 32;     // stride byte offset
-  d |= (uint64_t)1 << 46;               // descriptor version
-  d |= (uint64_t)2 << 61;               // SWIZZLE_128B
-  return d;
+// Shared-memory matrix descriptor of a K-major operand with 128-byte swizzle (rows 128 bytes apart,
+// groups of eight rows 1024 bytes apart, descriptor version 1), split into its address field (low
+// word: smem address / 16 in the low 14 bits, leading byte offset 1) and the constant rest, so that
+// stepping through a tile is one integer add.
+__device__ __forceinline__ uint32_t umma_desc_lo(uint32_t addr) { return ((addr >> 4) & 0x3fffu) | (1u << 16); }
+__device__ __forceinline__ uint64_t umma_desc_from_lo(uint32_t lo) {
+  constexpr uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+  return ((uint64_t)hi << 32) | lo;
 }
 
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t accumulate) {
@@ -204,34 +237,139 @@ __device__ __forceinline__ int ld_acquire(const int* p) {
   return v;
 }
 
+// One of a CTA's two streams of runs: run m of the stream is global run blockIdx.x + m * gridDim.x - shift.
+struct RunStream {
+  int m, k, tr, chunk, ric, u, g, head0, heads;
+  bool done;
+  __device__ void init() { m = 0, k = 0, tr = 0, chunk = -1, ric = 0, u = 0, g = 0, head0 = 0, heads = 1, done = false; }
+  // Moves to run m (or the next one that exists) and works out where its chunk lives.
+  __device__ void next_run(const TcArgs& a, int shift) {
+    int rho;
+    for (;; ++m) {
+      rho = (int)blockIdx.x + m * (int)gridDim.x - shift;
+      if (rho >= a.NR) {
+        done = true, tr = 0;
+        return;
+      }
+      if (rho >= 0) break;
+    }
+    const int c = rho / a.RPC;
+    ric = rho - c * a.RPC;
+    tr = min(a.run, a.T - ric * a.run);
+    k = 0;
+    if (c != chunk) {
+      chunk = c;
+      const int per_unit = a.Hkv * a.RB;
+      u = c / per_unit;
+      const int g_rb = c - u * per_unit;
+      g = g_rb / a.RB;
+      const int rb = g_rb - g * a.RB;
+      head0 = g * a.G + rb * a.hpb;
+      heads = min(a.hpb, a.G - rb * a.hpb);
+    }
+  }
+};
+
 // ------------------------------------------------------------------------------------ shared memory
 struct __align__(1024) Smem {
   uint8_t k[kStages][kTileBytes];  // K tiles: two 64-column halves of [128 rows][128 bytes], swizzled
   uint8_t q[2][kTileBytes];        // query rows of the P1 stream's chunk and of the P2 stream's chunk
-  float bias[kBiasSlots][kTile];   // row biases (max + log2 sum) of the P2 tile in flight
-  uint64_t full[kStages], empty[kStages], tmem_full[kTmemBufs], tmem_empty[kTmemBufs];
+  float nbias[kBiasBufs][kTile];   // negated row biases -(max + log2 sum) of the P2 stream's recent chunks
+  Desc desc[kRing];
+  // full[j % kFullBars] says sub-item j's K tile has landed.  There are two barriers per K stage so that
+  // each of the two MMA threads (even / odd j) sees every phase of the barriers it waits on: a parity wait
+  // is only sound for a waiter that never skips a phase.
+  uint64_t full[kFullBars], empty[kStages], tmem_full[kTmemBufs], tmem_empty[kTmemBufs];
+  uint64_t q_full[2];              // a stream's Q rows have landed (both MMA threads wait on it)
   uint32_t tmem_base;
   int abort_flag;
+  int p2_ready_gen;   // scout -> producer: biases of P2 chunk generations up to this one are staged
+  int gen_started;    // producer -> scout: latest P2 chunk generation whose first tile was issued ...
+  int gen_start_j[kBiasBufs];  // ... and the sub-item index of that first tile, per generation % kBiasBufs
+  int prod_j;         // producer -> scout: index of the sub-item being issued
 };
+static_assert(sizeof(Smem) <= 232448, "shared memory of one CTA");
+
+// One 32-column slice of an accumulator tile, with the causal / end-of-sequence mask of a P1 row
+// applied when the tile reaches past the prefix: keys t > limit are hidden (-inf).
+__device__ __forceinline__ void load_logits(uint32_t taddr, float (&v)[32], bool tail, int tbase, int limit) {
+  tmem_ld32(taddr, v);
+  if (tail) {
+#pragma unroll
+    for (int jj = 0; jj < 32; ++jj)
+      if (tbase + jj > limit) v[jj] = -INFINITY;
+  }
+}
+
+// Merge of `count` partial (max, sum) pairs of one row, 1 KB apart, in slot order.
+__device__ __forceinline__ float2 merge_pairs(const float2* p, int count) {
+  float m = kMinRowMax, l = 0.f;
+  int sl = 0;
+  for (; sl + 32 <= count; sl += 32) {  // all loads of a batch in flight together
+    float2 pr[32];
+#pragma unroll
+    for (int e = 0; e < 32; ++e) pr[e] = __ldcg(p + (int64_t)(sl + e) * kTile);
+    float bm = pr[0].x;
+#pragma unroll
+    for (int e = 1; e < 32; ++e) bm = fmaxf(bm, pr[e].x);
+    const float mn = fmaxf(m, bm);
+    float acc = l * ex2(m - mn);
+#pragma unroll
+    for (int e = 0; e < 32; ++e) acc += pr[e].y * ex2(pr[e].x - mn);
+    m = mn, l = acc;
+  }
+  for (; sl < count; ++sl) {
+    const float2 pr = __ldcg(p + (int64_t)sl * kTile);
+    const float mn = fmaxf(m, pr.x);
+    l = l * ex2(m - mn) + pr.y * ex2(pr.x - mn);
+    m = mn;
+  }
+  return make_float2(m, l);
+}
+
+// Bounded wait on a flag in shared memory written by another warp of the CTA.
+template <typename Pred>
+__device__ __forceinline__ bool wait_flag(Pred pred, unsigned sleep_ns, volatile int* abort_flag, int* status, int code) {
+  const unsigned long long t0 = global_ns();
+  for (int it = 1; !pred(); ++it) {
+    __nanosleep(sleep_ns);
+    if ((it & 63) == 0) {
+      if (*abort_flag) return false;
+      if (global_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        atomicCAS(status, 0, code);
+        return false;
+      }
+    }
+  }
+  return true;
+}
 
 template <int W>
 __global__ void __launch_bounds__(kThreads, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map, TcArgs a) {
-  extern __shared__ uint8_t smem_raw[];
-  Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  if (smem_u32(smem_raw) & 1023u) {  // the swizzled tiles need 1024-byte alignment; never seen, but checked
+    if (threadIdx.x == 0) atomicCAS(a.status, 0, 41);
+    return;
+  }
+  Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &sm.abort_flag;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(smem_u32(&sm.full[s]), 1);
-      mbar_init(smem_u32(&sm.empty[s]), 1);
-    }
+    for (int s = 0; s < kStages; ++s) mbar_init(smem_u32(&sm.empty[s]), 1);
+    for (int s = 0; s < kFullBars; ++s) mbar_init(smem_u32(&sm.full[s]), 1);
     for (int b = 0; b < kTmemBufs; ++b) {
       mbar_init(smem_u32(&sm.tmem_full[b]), 1);
       mbar_init(smem_u32(&sm.tmem_empty[b]), 4);
     }
+    mbar_init(smem_u32(&sm.q_full[0]), 1);
+    mbar_init(smem_u32(&sm.q_full[1]), 1);
     sm.abort_flag = 0;
+    sm.p2_ready_gen = 0;
+    sm.gen_started = 0;
+    sm.prod_j = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -244,235 +382,326 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   tc_fence_after();
   const uint32_t tmem_base = sm.tmem_base;
 
-  Sched sched(blockIdx.x, gridDim.x);
-  SubItem s;
-  int j = 0;
-
   if (warp == 0) {
-    // ================================================================= TMA producer
-    int q_chunk[2] = {-1, -1}, q_last[2] = {-1000, -1000};
-    float4 bias_reg = make_float4(0.f, 0.f, 0.f, 0.f);
-    bool ok = true;
-    while (ok && sched.next(a, s)) {
-      const int stage = j % kStages;
-      const bool reload = s.chunk != q_chunk[s.type];
-      if (lane == 0) {
-        ok = mbar_wait(smem_u32(&sm.empty[stage]), ((j / kStages) & 1) ^ 1, abort_flag, a.status, 11);
-        if (ok && reload) {
-          const int jl = q_last[s.type];
-          if (jl >= 0 && j - jl < kStages)  // the MMAs that read the old rows must have completed
-            ok = mbar_wait(smem_u32(&sm.empty[jl % kStages]), (jl / kStages) & 1, abort_flag, a.status, 12);
-          if (ok && s.type == 1) {  // the chunk's row statistics must be final
-            const unsigned long long t0 = global_ns();
-            int it = 0;
-            while (ld_acquire(a.ready + s.chunk) < 4) {
-              __nanosleep(64);
-              if ((++it & 63) == 0) {
-                if (*abort_flag) {
-                  ok = false;
-                  break;
-                }
-                if (global_ns() - t0 > kWaitLimitNs) {
-                  *abort_flag = 1;
-                  atomicCAS(a.status, 0, 13);
-                  ok = false;
-                  break;
-                }
+    // ================================================================= producer: schedule + TMA (one thread)
+    if (lane == 0) {
+      RunStream st0, st1;  // the P1 stream and the P2 stream
+      st0.init(), st1.init();
+      st0.next_run(a, 0), st1.next_run(a, a.DR);
+      int q_chunk0 = -1, q_chunk1 = -1;      // chunk whose rows each stream's Q buffer holds
+      // last even and last odd sub-item that read each stream's Q buffer (one per MMA thread)
+      int q_last0e = -1000, q_last0o = -1000, q_last1e = -1000, q_last1o = -1000;
+      int q_loads0 = 0, q_loads1 = 0;        // loads into each stream's Q buffer so far
+      int gen = 0;  // P2 chunks entered so far; biases of generation e live in nbias[e % kBiasBufs]
+      const uint64_t pol_q = policy_evict_last();
+      const uint64_t pol_k0 = a.hints ? policy_evict_last() : policy_evict_normal();
+      const uint64_t pol_k1 = a.hints ? policy_evict_first() : policy_evict_normal();
+      bool ok = true;
+      int j = 0;
+      // Issues the next tile of a stream as sub-item j (ty is a compile-time constant at both call sites).
+      auto issue = [&](RunStream& r, const int ty, int& q_chunk, int& q_last_e, int& q_last_o, int& q_loads,
+                       const uint64_t pol_k) {
+        const int stage = j % kStages;
+        const uint32_t bar = smem_u32(&sm.full[j % kFullBars]);
+        int4* d = reinterpret_cast<int4*>(&sm.desc[j % kRing]);
+        const bool reload = r.chunk != q_chunk;
+        if (reload) {
+          // The MMAs that read the stream's old rows must have completed, those of either MMA thread (the
+          // two complete independently, and a thread still waiting for the old rows' barrier phase must not
+          // be overtaken by the next load).  The wait on this sub-item's K stage covers sub-items up to
+          // j - kStages; a younger reader needs its own stage's barrier.
+          if (q_last_e > j - kStages)
+            ok = mbar_wait(smem_u32(&sm.empty[q_last_e % kStages]), (q_last_e / kStages) & 1, abort_flag, a.status,
+                           12 | (j << 8));
+          if (ok && q_last_o > j - kStages)
+            ok = mbar_wait(smem_u32(&sm.empty[q_last_o % kStages]), (q_last_o / kStages) & 1, abort_flag, a.status,
+                           12 | (j << 8));
+          if (!ok) return;
+          ++q_loads;
+          q_chunk = r.chunk;
+          if (ty == kP2) {
+            ++gen;
+            *(volatile int*)&sm.gen_start_j[gen % kBiasBufs] = j;
+            __threadfence_block();
+            *(volatile int*)&sm.gen_started = gen;
+          }
+        }
+        if (j & 1) q_last_o = j;
+        else q_last_e = j;
+        const int tile = r.ric * a.run + r.k;
+        // the n-th load of a stream's rows (n = 0, 1, ...) completes phase n of its barrier: wait for parity n & 1
+        const int q_phase = (q_loads - 1) & 1;
+        d[0] = make_int4(ty | (q_phase << 9), r.chunk, tile, (r.k + 2 >= r.tr) ? r.ric * a.ppr + (r.k & 1) : -1);
+        d[1] = make_int4(r.k < 2, r.u * a.H + r.head0, r.heads, gen % kBiasBufs);
+        mbar_arrive_expect_tx(bar, kTileBytes);
+        if (reload) {
+          const uint32_t qbar = smem_u32(&sm.q_full[ty]);
+          mbar_arrive_expect_tx(qbar, a.q_bytes);
+          tma_load_5d(&q_map, smem_u32(sm.q[ty]), qbar, 0, 0, r.head0, 0, r.u, pol_q);
+          if (a.q_split) tma_load_5d(&q_map, smem_u32(sm.q[ty]) + kHalfBytes, qbar, 0, 0, r.head0, 1, r.u, pol_q);
+        }
+        tma_load_5d(&k_map, smem_u32(sm.k[stage]), bar, 0, tile * kTile, 0, r.g, r.u, pol_k);
+        TC_TRACE(1, j);
+        if (++r.k == r.tr) {
+          ++r.m;
+          r.next_run(a, ty == kP1 ? 0 : a.DR);
+        }
+      };
+      while (ok && !(st0.done && st1.done)) {
+#pragma unroll
+        for (int slot = 0; slot < 2; ++slot, ++j) {
+          // Even slots carry the P1 stream while it lasts; P2 tiles take the odd slots, never ahead of
+          // the P1 tile they are paired with, and both slots once P1 has ended.
+          int ty = kNop;
+          if (slot == 0 && !st0.done) {
+            ty = kP1;
+          } else if (!st1.done && (st0.done || st1.m < st0.m || (st1.m == st0.m && st1.k < st0.k))) {
+            ty = kP2;
+            if (st1.k == 0 && st1.chunk != q_chunk1) {
+              // a new chunk: its biases must have been staged by the scout warp
+              if (*(volatile int*)&sm.p2_ready_gen < gen + 1) {
+                ty = kNop;
+                if (st0.done) __nanosleep(100);
+                if (*abort_flag) ok = false;
+              } else {
+                __threadfence_block();
               }
             }
           }
+          ok = ok && mbar_wait(smem_u32(&sm.empty[j % kStages]), ((j / kStages) & 1) ^ 1, abort_flag, a.status,
+                               11 | (j << 8));
+          TC_TRACE(0, j);
+          if (!ok) break;
+          *(volatile int*)&sm.prod_j = j;
+          if (ty == kP1) {
+            issue(st0, kP1, q_chunk0, q_last0e, q_last0o, q_loads0, pol_k0);
+          } else if (ty == kP2) {
+            issue(st1, kP2, q_chunk1, q_last1e, q_last1o, q_loads1, pol_k1);
+          } else {
+            sm.desc[j % kRing].type = kNop;
+            mbar_arrive(smem_u32(&sm.full[j % kFullBars]));
+          }
+          if (!ok) break;
         }
+      }
+      // one stop marker per consumer group
+      for (int e = 0; e < kTmemBufs && ok; ++e, ++j) {
+        ok = mbar_wait(smem_u32(&sm.empty[j % kStages]), ((j / kStages) & 1) ^ 1, abort_flag, a.status, 14 | (j << 8));
+        if (ok) {
+          sm.desc[j % kRing].type = kStop;
+          mbar_arrive(smem_u32(&sm.full[j % kFullBars]));
+        }
+      }
+      if (!ok) {
+        // give copies in flight time to land before the CTA's shared memory goes away
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+      }
+    }
+  } else if (warp == kScoutWarp) {
+    // ================================================================= scout: stages the biases of the P2 chunks
+    int gen = 0, prev_chunk = -1;
+    bool ok = true;
+    for (int m = 0; ok; ++m) {
+      const int rho = (int)blockIdx.x + m * (int)gridDim.x - a.DR;
+      if (rho >= a.NR) break;
+      if (rho < 0) continue;
+      const int c = rho / a.RPC;
+      if (c == prev_chunk) continue;
+      prev_chunk = c;
+      ++gen;
+      if (lane == 0) {
+        // nbias[gen % kBiasBufs] last served generation gen - kBiasBufs, whose tiles all precede the first
+        // tile of generation gen - kBiasBufs + 1; a tile's readers are done once the producer has got
+        // kStages + kTmemBufs sub-items past it (it waits for the K stage of sub-item j - kStages to be free,
+        // whose MMA waited for the TMEM buffer of sub-item j - kStages - kTmemBufs).
+        if (gen > kBiasBufs) {
+          const int g1 = gen - kBiasBufs + 1;
+          ok = wait_flag(
+              [&] {
+                if (*(volatile int*)&sm.gen_started < g1) return false;
+                __threadfence_block();
+                return *(volatile int*)&sm.prod_j >=
+                       *(volatile int*)&sm.gen_start_j[g1 % kBiasBufs] + kStages + kTmemBufs - 1;
+              },
+              200, abort_flag, a.status, 15);
+        }
+        // the chunk's row statistics must be final
+        ok = ok && wait_flag([&] { return ld_acquire(a.ready + c) >= 4; }, 100, abort_flag, a.status, 13);
       }
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
       if (!ok) break;
-      if (s.type == 1) {
-        if (reload) {
-          const float2* st = a.stat + (int64_t)s.chunk * kTile + 4 * lane;
-          const float2 s0 = __ldcg(st), s1 = __ldcg(st + 1), s2 = __ldcg(st + 2), s3 = __ldcg(st + 3);
-          bias_reg = make_float4(s0.y, s1.y, s2.y, s3.y);
-        }
-        reinterpret_cast<float4*>(sm.bias[j % kBiasSlots])[lane] = bias_reg;
-        __syncwarp();
-      }
+      const float2* stp = a.stat + (int64_t)c * kTile + 4 * lane;
+      const float2 s0 = __ldcg(stp), s1 = __ldcg(stp + 1), s2 = __ldcg(stp + 2), s3 = __ldcg(stp + 3);
+      reinterpret_cast<float4*>(sm.nbias[gen % kBiasBufs])[lane] = make_float4(-s0.y, -s1.y, -s2.y, -s3.y);
+      __syncwarp();
       if (lane == 0) {
-        const int g_rb = s.chunk % (a.Hkv * a.RB);
-        const int u = s.chunk / (a.Hkv * a.RB), g = g_rb / a.RB, rb = g_rb % a.RB;
-        const uint32_t bar = smem_u32(&sm.full[stage]);
-        mbar_arrive_expect_tx(bar, kTileBytes + (reload ? 2 * a.q_half_bytes : 0));
-        if (reload) {
-          const uint32_t qdst = smem_u32(sm.q[s.type]);
-          const int head0 = g * a.G + rb * a.hpb;
-          tma_load_4d(&q_map, qdst, bar, 0, 0, head0, u);
-          tma_load_4d(&q_map, qdst + kHalfBytes, bar, 64, 0, head0, u);
-        }
-        const uint32_t kdst = smem_u32(sm.k[stage]);
-        tma_load_4d(&k_map, kdst, bar, 0, s.tile * kTile, g, u);
-        tma_load_4d(&k_map, kdst + kHalfBytes, bar, 64, s.tile * kTile, g, u);
+        __threadfence_block();
+        *(volatile int*)&sm.p2_ready_gen = gen;
       }
-      q_chunk[s.type] = s.chunk;
-      q_last[s.type] = j;
-      ++j;
     }
-    if (!ok && lane == 0) {
-      // give copies in flight time to land before the CTA's shared memory goes away
-      for (int i = 0; i < 200; ++i) __nanosleep(1000);
-    }
-  } else if (warp == 1) {
-    // ================================================================= MMA issuer
-    bool ok = true;
-    while (ok && sched.next(a, s)) {
-      const int stage = j % kStages, buf = j % kTmemBufs;
-      if (lane == 0) {
-        ok = mbar_wait(smem_u32(&sm.full[stage]), (j / kStages) & 1, abort_flag, a.status, 21) &&
-             mbar_wait(smem_u32(&sm.tmem_empty[buf]), ((j / kTmemBufs) & 1) ^ 1, abort_flag, a.status, 22);
-        if (ok) {
+  } else if (warp == 1 || warp == kMma2Warp) {
+    // ================================================================= MMA issuers
+    // Two threads take turns (even / odd sub-items), so that one waits and sets up while the other's
+    // instructions drain into the tensor pipe.  tcgen05.commit tracks the issuing thread's own MMAs.
+    if (lane == 0) {
+      const uint32_t k_lo = umma_desc_lo(smem_u32(sm.k[0])), q_lo = umma_desc_lo(smem_u32(sm.q[0]));
+      bool ok = true;
+      int stops = 0;
+      for (int j = warp == 1 ? 0 : 1; ok && stops < kTmemBufs / 2; j += 2) {
+        const int stage = j % kStages, buf = j % kTmemBufs;
+        ok = mbar_wait(smem_u32(&sm.full[j % kFullBars]), (j / kFullBars) & 1, abort_flag, a.status, 21 | (j << 8));
+        TC_TRACE(2, j);
+        if (!ok) break;
+        const int tq = sm.desc[j % kRing].type;
+        const int type = tq & 0xff;
+        ok = mbar_wait(smem_u32(&sm.tmem_empty[buf]), ((j / kTmemBufs) & 1) ^ 1, abort_flag, a.status, 22 | (j << 8));
+        if (!ok) break;
+        if (type == kP1 || type == kP2) {
+          ok = mbar_wait(smem_u32(&sm.q_full[type]), (tq >> 9) & 1, abort_flag, a.status, 23 | (j << 8));
+          if (!ok) break;
           tc_fence_after();
-          const uint32_t kaddr = smem_u32(sm.k[stage]), qaddr = smem_u32(sm.q[s.type]);
-          const uint32_t a_addr = s.type == 0 ? qaddr : kaddr, b_addr = s.type == 0 ? kaddr : qaddr;
+          const uint32_t kd = k_lo + stage * (kTileBytes >> 4);
+          const uint32_t qd = q_lo + type * (kTileBytes >> 4);
+          const uint32_t a_lo = type == kP1 ? qd : kd, b_lo = type == kP1 ? kd : qd;
           const uint32_t d = tmem_base + buf * kTile;
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks) {
-            const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-            umma_bf16(d, umma_desc(a_addr + off), umma_desc(b_addr + off), ks > 0 ? 1u : 0u);
+            const uint32_t off = ((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4;
+            umma_bf16(d, umma_desc_from_lo(a_lo + off), umma_desc_from_lo(b_lo + off), ks > 0 ? 1u : 0u);
           }
           umma_commit(smem_u32(&sm.empty[stage]));
           umma_commit(smem_u32(&sm.tmem_full[buf]));
+          TC_TRACE(3, j);
+        } else {
+          stops += type == kStop;
+          mbar_arrive(smem_u32(&sm.empty[stage]));
+          mbar_arrive(smem_u32(&sm.tmem_full[buf]));
         }
       }
-      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-      ++j;
     }
-  } else {
+  } else if (warp < 2 + kConsumerWarps) {
     // ================================================================= consumers
-    const int cw = warp - 2, set = cw >> 2, quad = warp & 3;
+    const int group = (warp - 2) >> 2, quad = warp & 3;
     const int row = quad * 32 + lane;  // TMEM lane: query row (P1) or key within the tile (P2)
-    float m_run = -INFINITY, l_run = 0.f;
-    bool ok = true;
-    while (ok && sched.next(a, s)) {
-      if ((j & 1) != set) {
-        ++j;
+    const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + group * kTile;
+    const uint32_t bar_full = smem_u32(&sm.tmem_full[group]), bar_empty = smem_u32(&sm.tmem_empty[group]);
+    float m_run = kMinRowMax, l_run = 0.f;
+    for (int j = group;; j += kTmemBufs) {
+      bool ok = mbar_wait(bar_full, (j / kTmemBufs) & 1, abort_flag, a.status, 31 | (j << 8));
+      ok = __all_sync(0xffffffffu, ok);
+      if (quad == 0 && lane == 0) TC_TRACE(4, j);
+      if (!ok) break;
+      Desc d = sm.desc[j % kRing];
+      d.type &= 0xff;
+      if (d.type == kStop) break;
+      if (d.type == kNop) {
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_empty);
         continue;
       }
-      const int buf = j % kTmemBufs;
-      ok = mbar_wait(smem_u32(&sm.tmem_full[buf]), (j / kTmemBufs) & 1, abort_flag, a.status, 31);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
       tc_fence_after();
-      const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * kTile;
-      const int t0 = s.tile * kTile;
+      const int t0 = d.tile * kTile;
       const bool tail = t0 + kTile > a.n;  // tile touches the window keys or the end of the sequence
 
-      if (s.type == 0) {
+      if (d.type == kP1) {
         // ---------------------------------------------------------- P1: running (max, sum) of this row
-        if (s.k < 2) m_run = -INFINITY, l_run = 0.f;
-        const int i = row % W;
+        if (d.first) m_run = kMinRowMax, l_run = 0.f;
+        const int limit = a.n + row % W;   // last key this window row sees
+        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll 1
         for (int cc = 0; cc < 4; ++cc) {
           float v[32];
-          tmem_ld32(taddr + cc * 32, v);
+          load_logits(taddr + cc * 32, v, tail, t0 + cc * 32, limit);
+#pragma unroll
+          for (int jj = 0; jj < 32; ++jj) mx[jj & 3] = fmaxf(mx[jj & 3], v[jj]);
+        }
+        const float m_new = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * kScale, m_run);
+        const float negm = -m_new;
+        float sum[4] = {l_run * ex2(m_run - m_new), 0.f, 0.f, 0.f};
+#pragma unroll 1
+        for (int cc = 0; cc < 4; ++cc) {
+          float v[32];
+          load_logits(taddr + cc * 32, v, tail, t0 + cc * 32, limit);
           if (cc == 3) {
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&sm.tmem_empty[buf]));
+            if (lane == 0) mbar_arrive(bar_empty);
           }
-          if (tail) {
 #pragma unroll
-            for (int jj = 0; jj < 32; ++jj) {
-              const int t = t0 + cc * 32 + jj;
-              if (t >= a.L || t > a.n + i) v[jj] = -INFINITY;
-            }
-          }
-          float cmax = v[0];
-#pragma unroll
-          for (int jj = 1; jj < 32; ++jj) cmax = fmaxf(cmax, v[jj]);
-          const float m_new = fmaxf(m_run, cmax * kScale);
-          if (m_new != -INFINITY) {
-            float acc = 0.f;
-#pragma unroll
-            for (int jj = 0; jj < 32; ++jj) acc += ex2(fmaf(v[jj], kScale, -m_new));
-            l_run = l_run * ex2(m_run - m_new) + acc;
-            m_run = m_new;
-          }
+          for (int jj = 0; jj < 32; ++jj) sum[jj & 3] += ex2(fmaf(v[jj], kScale, negm));
         }
-        if (s.k + 2 >= s.tr) {
-          // this warp's last tile of the run: publish the partial pair; the last warp of the chunk's
+        l_run = (sum[0] + sum[1]) + (sum[2] + sum[3]);
+        m_run = m_new;
+        if (d.part_slot >= 0) {
+          // this group's last tile of the run: publish the pair; the last warp of the chunk's
           // quadrant merges all of them in slot order
-          const int slot = s.run_in_chunk * 2 + (s.k & 1);
-          a.part[((int64_t)s.chunk * (2 * a.RPC) + slot) * kTile + row] = make_float2(m_run, l_run);
+          a.part[((int64_t)d.chunk * (a.ppr * a.RPC) + d.part_slot) * kTile + row] = make_float2(m_run, l_run);
           __threadfence();
           __syncwarp();
           int prev = 0;
-          if (lane == 0) prev = atomicAdd(a.done + s.chunk * 4 + quad, 1);
+          if (lane == 0) prev = atomicAdd(a.done + d.chunk * 4 + quad, 1);
           prev = __shfl_sync(0xffffffffu, prev, 0);
           if (prev + 1 == a.expected) {
             __threadfence();
-            const float2* p = a.part + (int64_t)s.chunk * (2 * a.RPC) * kTile + row;
-            float m = -INFINITY;
-            for (int sl = 0; sl < a.expected; ++sl) m = fmaxf(m, __ldcg(p + (int64_t)sl * kTile).x);
-            float l = 0.f;
-            for (int sl = 0; sl < a.expected; ++sl) {
-              const float2 pr = __ldcg(p + (int64_t)sl * kTile);
-              if (pr.y > 0.f) l += pr.y * ex2(pr.x - m);
-            }
-            a.stat[(int64_t)s.chunk * kTile + row] = make_float2(m, m + log2f(l));
+            const float2 ml = merge_pairs(a.part + (int64_t)d.chunk * (a.ppr * a.RPC) * kTile + row, a.expected);
+            a.stat[(int64_t)d.chunk * kTile + row] = make_float2(ml.x, ml.x + log2f(ml.y));
             __threadfence();
             __syncwarp();
-            if (lane == 0) atomicAdd(a.ready + s.chunk, 1);
+            if (lane == 0) atomicAdd(a.ready + d.chunk, 1);
           }
         }
       } else {
         // ---------------------------------------------------------- P2: column sums of this key
         const int t = t0 + row;
-        const float* bias = sm.bias[j % kBiasSlots];
-        const int g_rb = s.chunk % (a.Hkv * a.RB);
-        const int u = s.chunk / (a.Hkv * a.RB), g = g_rb / a.RB, rb = g_rb % a.RB;
-        constexpr int kHeadsPerChunk = W >= 32 ? 1 : 32 / W;  // heads inside one 32-row TMEM load
+        const float* nb = sm.nbias[d.nbias_buf];
+        constexpr int kHeadsPerSlice = W >= 32 ? 1 : 32 / W;  // heads inside one 32-row TMEM load
+        float* out = a.csum + (int64_t)d.head0 * a.L + t;
         float head_acc = 0.f;
 #pragma unroll 1
         for (int cc = 0; cc < 4; ++cc) {
           float v[32];
           tmem_ld32(taddr + cc * 32, v);
-          float acc[kHeadsPerChunk];
+          float acc[kHeadsPerSlice][2];
 #pragma unroll
-          for (int hh = 0; hh < kHeadsPerChunk; ++hh) acc[hh] = 0.f;
+          for (int hh = 0; hh < kHeadsPerSlice; ++hh) acc[hh][0] = acc[hh][1] = 0.f;
 #pragma unroll
           for (int j4 = 0; j4 < 8; ++j4) {
-            const float4 b4 = reinterpret_cast<const float4*>(bias)[cc * 8 + j4];
+            const float4 b4 = reinterpret_cast<const float4*>(nb)[cc * 8 + j4];
             const float bb[4] = {b4.x, b4.y, b4.z, b4.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
               const int jj = j4 * 4 + e;
-              float p = ex2(fmaf(v[jj], kScale, -bb[e]));
+              float p = ex2(fmaf(v[jj], kScale, bb[e]));
               if (tail) {
                 const int i = (cc * 32 + jj) % W;
                 if (t > a.n + i) p = 0.f;
               }
-              acc[W >= 32 ? 0 : jj / W] += p;
+              acc[W >= 32 ? 0 : jj / W][e & 1] += p;
             }
           }
           if (cc == 3) {  // all bias reads and TMEM loads of this sub-item are done
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&sm.tmem_empty[buf]));
+            if (lane == 0) mbar_arrive(bar_empty);
           }
           if (W >= 32) {
-            head_acc += acc[0];
+            head_acc += acc[0][0] + acc[0][1];
             const int rows_done = (cc + 1) * 32;
             if (rows_done % W == 0) {
-              const int hl = rb * a.hpb + rows_done / W - 1;
-              if (hl < a.G && t < a.L) a.csum[((int64_t)u * a.H + g * a.G + hl) * a.L + t] = head_acc;
+              const int hl = rows_done / W - 1;
+              if (hl < d.n_heads && t < a.L) out[(int64_t)hl * a.L] = head_acc;
               head_acc = 0.f;
             }
           } else {
 #pragma unroll
-            for (int hh = 0; hh < kHeadsPerChunk; ++hh) {
-              const int hl = rb * a.hpb + cc * kHeadsPerChunk + hh;
-              if (hl < a.G && t < a.L) a.csum[((int64_t)u * a.H + g * a.G + hl) * a.L + t] = acc[hh];
+            for (int hh = 0; hh < kHeadsPerSlice; ++hh) {
+              const int hl = cc * kHeadsPerSlice + hh;
+              if (hl < d.n_heads && t < a.L) out[(int64_t)hl * a.L] = acc[hh][0] + acc[hh][1];
             }
           }
         }
       }
-      ++j;
+      if (quad == 0 && lane == 0) TC_TRACE(5, j);
     }
   }
 
@@ -502,27 +731,27 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// bf16 tensor [d3][d2][d1][128] with element strides (s1, s2, s3); box [1][b2][b1][64], 128-byte swizzle.
-bool make_map(CUtensorMap* map, const void* base, uint64_t d1, uint64_t d2, uint64_t d3, int64_t s1, int64_t s2,
-              int64_t s3, uint32_t b1, uint32_t b2) {
+// Rank-5 bf16 tensor map whose innermost dimension is one 64-element half of a 128-element row and
+// one of whose outer dimensions selects the half (stride 128 bytes): a box that spans both halves lands
+// in shared memory as two [rows][64] blocks, which is the 128-byte-swizzled K-major operand layout.
+bool make_map5(CUtensorMap* map, const void* base, const cuuint64_t (&dims)[5], const cuuint64_t (&strides)[4],
+               const cuuint32_t (&box)[5]) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
-  // a dimension of extent one may carry any stride; give it a legal one
-  if (d1 == 1 || s1 <= 0) s1 = kHeadDim;
-  if (d2 == 1 || s2 <= 0) s2 = s1 * (int64_t)d1;
-  if (d3 == 1 || s3 <= 0) s3 = s2 * (int64_t)d2;
-  const cuuint64_t dims[4] = {(cuuint64_t)kHeadDim, d1, d2, d3};
-  const cuuint64_t strides[3] = {(cuuint64_t)s1 * 2, (cuuint64_t)s2 * 2, (cuuint64_t)s3 * 2};
-  const cuuint32_t box[4] = {64, b1, b2, 1};
-  const cuuint32_t estr[4] = {1, 1, 1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+  const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// A dimension of extent one may carry any stride; give it a legal one (in bytes).
+cuuint64_t legal_stride(uint64_t extent, int64_t stride_elems, cuuint64_t fallback_bytes) {
+  return (extent == 1 || stride_elems <= 0) ? fallback_bytes : (cuuint64_t)stride_elems * 2;
+}
+
 template <int W>
 cudaError_t launch_w(const CUtensorMap& qm, const CUtensorMap& km, const TcArgs& a, int grid, cudaStream_t st) {
-  const size_t smem = sizeof(Smem) + 1024;
+  const size_t smem = sizeof(Smem);
   cudaError_t e = cudaFuncSetAttribute(score_tc_kernel<W>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
@@ -535,6 +764,12 @@ cudaError_t launch_w(const CUtensorMap& qm, const CUtensorMap& km, const TcArgs&
 }
 
 }  // namespace
+
+#ifdef CKV_TC_TRACE
+extern "C" __attribute__((visibility("default"))) int ckv_debug_tc_trace(long long* out) {
+  return cudaMemcpyFromSymbol(out, g_tc_trace, sizeof(long long) * 6 * 1024) != cudaSuccess;
+}
+#endif
 
 bool score_tc_supported(const ckv_shape& s) {
   if (s.dtype != CKV_BF16) return false;
@@ -550,38 +785,67 @@ TcLayout tc_layout(const ckv_shape& s) {
   const int G = s.n_q_heads / s.n_kv_heads;
   t.RB = (G * s.window + kTile - 1) / kTile;
   t.T = (s.seq_len + kTile - 1) / kTile;
-  t.RPC = (t.T + kRun - 1) / kRun;
   t.C = (int64_t)s.n_units * s.n_kv_heads * t.RB;
-  t.part_bytes = (size_t)t.C * 2 * t.RPC * kTile * sizeof(float2);
+  t.part_bytes = (size_t)t.C * (t.T + 2) * kTile * sizeof(float2);  // at most T + 1 pairs per chunk
   t.stat_bytes = (size_t)t.C * kTile * sizeof(float2);
   t.flag_bytes = (size_t)t.C * 5 * sizeof(int);
   return t;
 }
 
+int set_tc_tunable(const char* name, int value) {
+  const std::string n(name);
+  if (n == "run_tiles" && value >= 1 && value <= 64) return g_run_tiles.exchange(value);
+  if (n == "lag_slack_pct" && value >= 0 && value <= 1000) return g_lag_slack_pct.exchange(value);
+  if (n == "l2_hints" && (value == 0 || value == 1)) return g_l2_hints.exchange(value);
+  return -1;
+}
+
 cudaError_t launch_score_tc(const ckv_shape& s, const void* q, const void* k, float* csum, void* part, void* stat,
                             int* flags, int* status, cudaStream_t st) {
   const TcLayout t = tc_layout(s);
-  if (t.C > (int64_t)1 << 24) return cudaErrorInvalidValue;
   TcArgs a{};
   a.Nu = s.n_units, a.H = s.n_q_heads, a.Hkv = s.n_kv_heads, a.G = a.H / a.Hkv, a.L = s.seq_len, a.W = s.window;
   a.n = a.L - a.W;
-  a.RB = t.RB, a.hpb = kTile / a.W, a.T = t.T, a.RPC = t.RPC, a.C = (int)t.C;
+  a.RB = t.RB, a.hpb = kTile / a.W, a.T = t.T, a.C = (int)t.C;
+  a.run = g_run_tiles.load();
+  a.RPC = (a.T + a.run - 1) / a.run;
+  if (t.C * a.RPC > (int64_t)1 << 30) return cudaErrorInvalidValue;
   a.NR = a.C * a.RPC;
   int dev = 0, sms = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int grid = sms < a.NR ? sms : a.NR;
-  a.DR = a.RPC + 2 * grid;
-  const int t_last = a.T - (a.RPC - 1) * kRun;
-  a.expected = 2 * (a.RPC - 1) + (t_last < 2 ? t_last : 2);
+  a.DR = a.RPC + (int)(((int64_t)grid * g_lag_slack_pct.load() + 99) / 100);
+  const int t_last = a.T - (a.RPC - 1) * a.run;
+  a.ppr = a.run < 2 ? 1 : 2;
+  a.expected = (a.RPC - 1) * a.ppr + (t_last < 2 ? t_last : 2);
+  a.hints = g_l2_hints.load();
   const int hpb_box = a.hpb < a.H ? a.hpb : a.H;
-  a.q_half_bytes = 64u * 2u * (uint32_t)a.W * (uint32_t)hpb_box;
+  a.q_bytes = 2u * 64u * 2u * (uint32_t)a.W * (uint32_t)hpb_box;
+  a.q_split = hpb_box * a.W < kTile;  // a short box would pack its halves closer than the operand layout wants
   a.csum = csum, a.part = (float2*)part, a.stat = (float2*)stat;
   a.done = flags, a.ready = flags + 4 * a.C, a.status = status;
   CUtensorMap qm, km;
-  if (!make_map(&qm, q, a.W, a.H, a.Nu, s.q_stride_row, s.q_stride_head, s.q_stride_unit, a.W, hpb_box) ||
-      !make_map(&km, k, a.L, a.Hkv, a.Nu, s.kv_stride_tok, s.kv_stride_head, s.kv_stride_unit, kTile, 1))
-    return cudaErrorInvalidValue;
+  {
+    // Q: [unit][half][head][row][64]; box = one row block (hpb heads x W rows) x both halves
+    const cuuint64_t row_b = legal_stride(a.W, s.q_stride_row, kHeadDim * 2);
+    const cuuint64_t head_b = legal_stride(a.H, s.q_stride_head, row_b * a.W);
+    const cuuint64_t unit_b = legal_stride(a.Nu, s.q_stride_unit, head_b * a.H);
+    const cuuint64_t dims[5] = {64, (cuuint64_t)a.W, (cuuint64_t)a.H, 2, (cuuint64_t)a.Nu};
+    const cuuint64_t strides[4] = {row_b, head_b, 128, unit_b};
+    const cuuint32_t box[5] = {64, (cuuint32_t)a.W, (cuuint32_t)hpb_box, a.q_split ? 1u : 2u, 1};
+    if (!make_map5(&qm, q, dims, strides, box)) return cudaErrorInvalidValue;
+  }
+  {
+    // K: [unit][head][half][token][64]; box = 128 tokens x both halves
+    const cuuint64_t tok_b = legal_stride(a.L, s.kv_stride_tok, kHeadDim * 2);
+    const cuuint64_t head_b = legal_stride(a.Hkv, s.kv_stride_head, tok_b * a.L);
+    const cuuint64_t unit_b = legal_stride(a.Nu, s.kv_stride_unit, head_b * a.Hkv);
+    const cuuint64_t dims[5] = {64, (cuuint64_t)a.L, 2, (cuuint64_t)a.Hkv, (cuuint64_t)a.Nu};
+    const cuuint64_t strides[4] = {tok_b, 128, head_b, unit_b};
+    const cuuint32_t box[5] = {64, kTile, 2, 1, 1};
+    if (!make_map5(&km, k, dims, strides, box)) return cudaErrorInvalidValue;
+  }
   cudaError_t e = cudaMemsetAsync(flags, 0, t.flag_bytes, st);
   if (e != cudaSuccess) return e;
   if (a.W == 16) e = launch_w<16>(qm, km, a, grid, st);
