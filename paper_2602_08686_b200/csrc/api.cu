@@ -27,6 +27,12 @@ WsLayout ws_layout(const ckv_shape& s, const ckv_params&) {
   w.scores = o, o = align_up(o + Nu * Hkv * (n ? n : 1) * sizeof(float));
   w.bucket = o, o = align_up(o + Nu * sizeof(int32_t));
   w.entropy = o, o = align_up(o + Nu * sizeof(float));
+  {
+    const BudgetLayout b = budget_layout(s);
+    w.ent_part = o, o = align_up(o + b.ent_bytes);
+    w.cnt_part = o, o = align_up(o + b.cnt_bytes);
+    w.bud_done = o, o = align_up(o + b.done_bytes);
+  }
   if (s.dtype == CKV_BF16) {
     const TcLayout t = tc_layout(s);
     w.tc_part = o, o = align_up(o + t.part_bytes);
@@ -145,8 +151,10 @@ ckv_status ckv_budget(const ckv_shape* shape, const ckv_params* params, const fl
   CKV_TRY(check_params(shape, params));
   if (!all_aligned4({scores, colmass, sens, budgets, offsets, bucket, entropy})) return CKV_ERR_INVALID_ARG;
   CKV_TRY(check_ws(shape, params, ws, ws_bytes));
+  const WsLayout w = ws_layout(*shape, *params);
+  char* base = (char*)ws;
   CKV_CUDA(launch_budget(*shape, *params, scores, colmass, sens, budgets, offsets, bucket, entropy,
-                         (cudaStream_t)stream));
+                         base + w.ent_part, base + w.cnt_part, base + w.bud_done, (cudaStream_t)stream));
   return CKV_OK;
 }
 
@@ -189,7 +197,8 @@ ckv_status ckv_compress(const ckv_shape* shape, const ckv_params* params, const 
   int32_t* bucket = bucket_or_null ? bucket_or_null : reinterpret_cast<int32_t*>(base + w.bucket);
   float* entropy = entropy_or_null ? entropy_or_null : reinterpret_cast<float*>(base + w.entropy);
   CKV_TRY(score_impl(*shape, *params, q_win, k, head_w, scores, colmass, base, st));
-  CKV_CUDA(launch_budget(*shape, *params, scores, colmass, sens, budgets, offsets, bucket, entropy, st));
+  CKV_CUDA(launch_budget(*shape, *params, scores, colmass, sens, budgets, offsets, bucket, entropy,
+                         base + w.ent_part, base + w.cnt_part, base + w.bud_done, st));
   CKV_CUDA(launch_select(*shape, *params, scores, budgets, offsets, indices, st));
   CKV_CUDA(launch_gather(*shape, *params, k, v, indices, offsets, k_out, v_out, st));
   return CKV_OK;

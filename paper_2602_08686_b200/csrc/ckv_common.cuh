@@ -28,9 +28,19 @@ struct WsLayout {
   size_t tc_part;  // float2 [C, T+2, 128]     partial row statistics of the tensor-core scan
   size_t tc_stat;  // float2 [C, 128]          final row statistics per chunk
   size_t tc_flags; // int32 [C, 5]             completion counters and ready flags
+  size_t ent_part; // double [Nu, nblk]        entropy partials of the budget stage
+  size_t cnt_part; // int32 [Nu, Hkv, S]       candidate counts per slice
+  size_t bud_done; // int32 [Nu]               CTAs of the unit that have finished counting
   size_t total;
   int nblk;
 };
+
+// Scratch of the budget stage: entropy blocks per unit, score slices per KV head.
+struct BudgetLayout {
+  int nblk, S;
+  size_t ent_bytes, cnt_bytes, done_bytes;
+};
+BudgetLayout budget_layout(const ckv_shape& s);
 
 // Sizes of the tensor-core scan's scratch for a shape (chunks of 128 query rows x whole key range).
 struct TcLayout {
@@ -55,7 +65,7 @@ cudaError_t launch_epilogue(const ckv_shape& s, const ckv_params& p, const float
                             float* scores, float* colmass, cudaStream_t st);
 cudaError_t launch_budget(const ckv_shape& s, const ckv_params& p, const float* scores, const float* colmass,
                           const float* sens, int32_t* budgets, int32_t* offsets, int32_t* bucket, float* entropy,
-                          cudaStream_t st);
+                          void* ent_part, void* cnt_part, void* done, cudaStream_t st);
 cudaError_t launch_select(const ckv_shape& s, const ckv_params& p, const float* scores, const int32_t* budgets,
                           const int32_t* offsets, int32_t* indices, cudaStream_t st);
 cudaError_t launch_gather(const ckv_shape& s, const ckv_params& p, const void* k, const void* v,

@@ -85,10 +85,13 @@ struct TcArgs {
 // Optional event trace of one CTA (a profiling build defines CKV_TC_TRACE).
 #ifdef CKV_TC_TRACE
 __device__ long long g_tc_trace[6][1024];
+__device__ unsigned long long g_tc_count[8];  // slots, P1 tiles, P2 tiles, no-ops: not ready / pairing / other
 #define TC_TRACE(ev, jj) \
   do { if (blockIdx.x == 5 && (jj) < 1024) g_tc_trace[ev][jj] = clock64(); } while (0)
+#define TC_COUNT(i) atomicAdd(&g_tc_count[i], 1ull)
 #else
 #define TC_TRACE(ev, jj) do {} while (0)
+#define TC_COUNT(i) do {} while (0)
 #endif
 
 // What the producer tells the other warps about sub-item j (ring slot j % kRing).
@@ -461,6 +464,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
               // a new chunk: its biases must have been staged by the scout warp
               if (*(volatile int*)&sm.p2_ready_gen < gen + 1) {
                 ty = kNop;
+                TC_COUNT(3);
                 if (st0.done) __nanosleep(100);
                 if (*abort_flag) ok = false;
               } else {
@@ -472,6 +476,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
                                11 | (j << 8));
           TC_TRACE(0, j);
           if (!ok) break;
+          TC_COUNT(0);
+          if (ty == kNop && !st1.done) TC_COUNT(4);
+          if (ty != kNop) TC_COUNT(1 + ty);
           *(volatile int*)&sm.prod_j = j;
           if (ty == kP1) {
             issue(st0, kP1, q_chunk0, q_last0e, q_last0o, q_loads0, pol_k0);
@@ -766,6 +773,11 @@ cudaError_t launch_w(const CUtensorMap& qm, const CUtensorMap& km, const TcArgs&
 }  // namespace
 
 #ifdef CKV_TC_TRACE
+extern "C" __attribute__((visibility("default"))) int ckv_debug_tc_counts(unsigned long long* out, int reset) {
+  if (cudaMemcpyFromSymbol(out, g_tc_count, sizeof(g_tc_count)) != cudaSuccess) return 1;
+  unsigned long long z[8] = {};
+  return reset && cudaMemcpyToSymbol(g_tc_count, z, sizeof(z)) != cudaSuccess;
+}
 extern "C" __attribute__((visibility("default"))) int ckv_debug_tc_trace(long long* out) {
   return cudaMemcpyFromSymbol(out, g_tc_trace, sizeof(long long) * 6 * 1024) != cudaSuccess;
 }

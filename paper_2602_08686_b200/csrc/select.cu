@@ -2,12 +2,16 @@
 // key of the k-th largest score, then one ordered compaction writes the kept positions in
 // ascending order; equal scores are resolved toward the lowest index, and the observation window
 // is appended.  One CTA per (unit, KV head); integer work only, bit-exact and deterministic.
+// Thread i owns the contiguous positions [i*chunk, (i+1)*chunk); when a head's prefix fits
+// (chunk <= 32) the keys stay in registers for all four digit passes and the compaction.
 #include "ckv_common.cuh"
 
 namespace ckv {
 namespace {
 
 constexpr int kThreads = 1024;
+constexpr int kWarps = kThreads / 32;
+constexpr int kCache = 32;   // keys a thread can keep in registers
 
 // Order-preserving map from float bits to unsigned: larger float <=> larger key.
 __device__ __forceinline__ uint32_t key_of(float x) {
@@ -15,20 +19,23 @@ __device__ __forceinline__ uint32_t key_of(float x) {
   return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
+template <bool kCached>
 __global__ void __launch_bounds__(kThreads) select_kernel(ckv_shape s, const float* __restrict__ scores,
                                                           const int32_t* __restrict__ budgets,
                                                           const int32_t* __restrict__ offsets,
                                                           int32_t* __restrict__ indices) {
-  __shared__ int hist[256];
+  __shared__ int whist[kWarps][256];   // one histogram per warp: no contention between warps
+  __shared__ int suffix[256];
   __shared__ uint32_t sh_prefix;
   __shared__ int sh_want;
-  __shared__ int warp_gt[kThreads / 32], warp_eq[kThreads / 32];
+  __shared__ int warp_gt[kWarps], warp_eq[kWarps];
   const int Hkv = s.n_kv_heads, W = s.window, n = s.seq_len - W;
   const int u = blockIdx.x / Hkv, g = blockIdx.x % Hkv;
   const int e = budgets[(int64_t)u * Hkv + g] - W;
   const int64_t rows_per_unit = offsets[(int64_t)u * (Hkv + 1) + Hkv];
   int32_t* out = indices + (int64_t)u * rows_per_unit + offsets[(int64_t)u * (Hkv + 1) + g];
   const float* sc = scores + ((int64_t)u * Hkv + g) * n;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
   for (int i = threadIdx.x; i < W; i += kThreads) out[e + i] = n + i;
   if (e <= 0) return;
@@ -37,26 +44,74 @@ __global__ void __launch_bounds__(kThreads) select_kernel(ckv_shape s, const flo
     return;
   }
 
+  const int chunk = (n + kThreads - 1) / kThreads;
+  const int t0 = min(threadIdx.x * chunk, n), t1 = min(t0 + chunk, n);
+  uint32_t keys[kCached ? kCache : 1];
+  if (kCached) {
+#pragma unroll
+    for (int j = 0; j < kCache; ++j) keys[j] = (t0 + j < t1) ? key_of(sc[t0 + j]) : 0u;
+  }
+
   // radix select, 8 bits per pass from the top: after the loop `prefix` is the key of the e-th
   // largest score and `want` the number of scores equal to it that are kept
   uint32_t prefix = 0, mask = 0;
   int want = e;
   for (int shift = 24; shift >= 0; shift -= 8) {
-    if (threadIdx.x < 256) hist[threadIdx.x] = 0;
+    for (int i = lane; i < 256; i += 32) whist[warp][i] = 0;
+    __syncwarp();
+    // consecutive equal digits of a thread are added in one go (scores of one head share their top bits)
+    int run_bin = -1, run_cnt = 0;
+#pragma unroll
+    for (int j = 0; j < (kCached ? kCache : 1); ++j) {
+      if (kCached) {
+        if (t0 + j < t1 && (keys[j] & mask) == prefix) {
+          const int bin = (keys[j] >> shift) & 0xff;
+          if (bin == run_bin) {
+            ++run_cnt;
+          } else {
+            if (run_cnt) atomicAdd(&whist[warp][run_bin], run_cnt);
+            run_bin = bin, run_cnt = 1;
+          }
+        }
+      }
+    }
+    if (!kCached) {
+      for (int t = t0; t < t1; ++t) {
+        const uint32_t key = key_of(sc[t]);
+        if ((key & mask) == prefix) {
+          const int bin = (key >> shift) & 0xff;
+          if (bin == run_bin) {
+            ++run_cnt;
+          } else {
+            if (run_cnt) atomicAdd(&whist[warp][run_bin], run_cnt);
+            run_bin = bin, run_cnt = 1;
+          }
+        }
+      }
+    }
+    if (run_cnt) atomicAdd(&whist[warp][run_bin], run_cnt);
     __syncthreads();
-    for (int t = threadIdx.x; t < n; t += kThreads) {
-      const uint32_t key = key_of(sc[t]);
-      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 0xff], 1);
+    if (threadIdx.x < 256) {
+      int tot = 0;
+#pragma unroll 8
+      for (int w = 0; w < kWarps; ++w) tot += whist[w][threadIdx.x];
+      suffix[threadIdx.x] = tot;
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
-      int acc = 0, dgt = 255;
-      for (; dgt > 0; --dgt) {
-        if (acc + hist[dgt] >= want) break;
-        acc += hist[dgt];
+    // suffix[b] = number of matching keys whose digit is >= b
+    for (int o = 1; o < 256; o <<= 1) {
+      int add = 0;
+      if (threadIdx.x < 256 && threadIdx.x + o < 256) add = suffix[threadIdx.x + o];
+      __syncthreads();
+      if (threadIdx.x < 256) suffix[threadIdx.x] += add;
+      __syncthreads();
+    }
+    if (threadIdx.x < 256) {
+      const int here = suffix[threadIdx.x], above = threadIdx.x < 255 ? suffix[threadIdx.x + 1] : 0;
+      if (here >= want && above < want) {   // exactly one digit qualifies
+        sh_prefix = prefix | ((uint32_t)threadIdx.x << shift);
+        sh_want = want - above;
       }
-      sh_prefix = prefix | ((uint32_t)dgt << shift);
-      sh_want = want - acc;
     }
     __syncthreads();
     prefix = sh_prefix;
@@ -65,16 +120,19 @@ __global__ void __launch_bounds__(kThreads) select_kernel(ckv_shape s, const flo
     __syncthreads();
   }
 
-  // ordered compaction: thread i owns the contiguous positions [i*chunk, (i+1)*chunk)
-  const int chunk = (n + kThreads - 1) / kThreads;
-  const int t0 = min(threadIdx.x * chunk, n), t1 = min(t0 + chunk, n);
+  // ordered compaction
   int gt = 0, eq = 0;
-  for (int t = t0; t < t1; ++t) {
-    const uint32_t key = key_of(sc[t]);
-    gt += key > prefix;
-    eq += key == prefix;
+  if (kCached) {
+#pragma unroll
+    for (int j = 0; j < kCache; ++j)
+      if (t0 + j < t1) gt += keys[j] > prefix, eq += keys[j] == prefix;
+  } else {
+    for (int t = t0; t < t1; ++t) {
+      const uint32_t key = key_of(sc[t]);
+      gt += key > prefix;
+      eq += key == prefix;
+    }
   }
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   int gt_inc = gt, eq_inc = eq;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -96,8 +154,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(ckv_shape s, const flo
   }
   __syncthreads();
   int gt_before = warp_gt[warp] + gt_inc - gt, eq_before = warp_eq[warp] + eq_inc - eq;
-  for (int t = t0; t < t1; ++t) {
-    const uint32_t key = key_of(sc[t]);
+  auto place = [&](uint32_t key, int t) {
     if (key > prefix) {
       out[gt_before + min(eq_before, want)] = t;
       ++gt_before;
@@ -105,6 +162,13 @@ __global__ void __launch_bounds__(kThreads) select_kernel(ckv_shape s, const flo
       if (eq_before < want) out[gt_before + eq_before] = t;
       ++eq_before;
     }
+  };
+  if (kCached) {
+#pragma unroll
+    for (int j = 0; j < kCache; ++j)
+      if (t0 + j < t1) place(keys[j], t0 + j);
+  } else {
+    for (int t = t0; t < t1; ++t) place(key_of(sc[t]), t);
   }
 }
 
@@ -112,7 +176,12 @@ __global__ void __launch_bounds__(kThreads) select_kernel(ckv_shape s, const flo
 
 cudaError_t launch_select(const ckv_shape& s, const ckv_params&, const float* scores, const int32_t* budgets,
                           const int32_t* offsets, int32_t* indices, cudaStream_t st) {
-  select_kernel<<<s.n_units * s.n_kv_heads, kThreads, 0, st>>>(s, scores, budgets, offsets, indices);
+  const int n = s.seq_len - s.window;
+  const int grid = s.n_units * s.n_kv_heads;
+  if ((n + kThreads - 1) / kThreads <= kCache)
+    select_kernel<true><<<grid, kThreads, 0, st>>>(s, scores, budgets, offsets, indices);
+  else
+    select_kernel<false><<<grid, kThreads, 0, st>>>(s, scores, budgets, offsets, indices);
   count_launch();
   return cudaGetLastError();
 }
