@@ -191,9 +191,7 @@ ckv_status ckv_device_status(const void* ws, void* stream);
 int ckv_set_score_path(int path);
 
 /* Diagnostic knobs of the tensor-core scan's schedule (process-wide; results do not depend on them):
- *   "run_tiles"      key tiles per run, the unit CTAs take work in (1..64, default 4);
- *   "lag_slack_pct"  how far the second pass trails the first beyond one chunk, in percent of the
- *                    number of CTAs (0..1000, default 200);
+ *   "run_tiles"      key tiles per run, the unit CTAs take work in (1..64, default 8);
  *   "l2_hints"       1 (default): first-pass K loads ask L2 to keep their lines and second-pass loads
  *                    release them; 0: no hints.
  * Returns the previous value, or -1 for an unknown name or a value out of range. */

@@ -91,7 +91,7 @@ def ckv_set_score_path(path: int) -> int:
 
 
 def ckv_set_tunable(name: str, value: int) -> int:
-    """Schedule knob of the tensor-core scan ("run_tiles", "lag_slack_pct", "l2_hints"); returns the previous value."""
+    """Schedule knob of the tensor-core scan ("run_tiles", "l2_hints"); returns the previous value."""
     prev = int(lib().ckv_set_tunable(name.encode(), int(value)))
     if prev < 0:
         raise ValueError(f"unknown tunable or value out of range: {name}={value}")

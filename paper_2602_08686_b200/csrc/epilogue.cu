@@ -5,78 +5,131 @@
 namespace ckv {
 namespace {
 
-constexpr int kThreads = 256;   // positions per CTA
-constexpr int kMaxHalo = 7;     // pool_size <= 15
-constexpr int kHeadBatch = 8;   // heads staged in shared memory at a time
+constexpr int kThreads = 128;
+constexpr int kPerThread = 4;                    // consecutive positions per thread
+constexpr int kSpan = kThreads * kPerThread;     // positions per CTA
+constexpr int kHeadBatch = 8;                    // heads staged in shared memory at a time
 
-// One CTA owns 256 consecutive positions t of one unit and walks over all query heads:
+// One CTA owns kSpan consecutive positions t of one unit and walks over all query heads:
 //   scores[u,g,t] = max_{h in g} head_w[h] * pool((L/W) c_h)[t]   for t < n  (pooling never looks past n)
 //   colmass[u,t]  = sum_h c_h[t]                                    for t < L  (heads added in index order)
+// R is the pooling radius (window 2R + 1); AVG counts positions outside the prefix as zeros and divides
+// by the window size, MAX ignores them.
+template <int R, bool AVG>
 __global__ void __launch_bounds__(kThreads) pool_weight_max_mass(ckv_shape s, ckv_params p,
                                                                  const float* __restrict__ csum,
                                                                  const float* __restrict__ head_w,
                                                                  float* __restrict__ scores,
                                                                  float* __restrict__ colmass) {
-  __shared__ float tile[kHeadBatch][kThreads + 2 * kMaxHalo];
+  constexpr int kHalo = (R + 3) / 4 * 4;           // halo rounded up so that every thread's window is 16-byte aligned
+  constexpr int kWidth = kSpan + 2 * kHalo;        // staged positions t0 - kHalo .. t0 + kSpan + kHalo - 1
+  constexpr int kWin = kPerThread + 2 * kHalo;     // values a thread reads: c_h[tb - kHalo .. tb + 3 + kHalo]
+  __shared__ __align__(16) float tile[kHeadBatch][kWidth];
   const int L = s.seq_len, n = L - s.window, H = s.n_q_heads, G = H / s.n_kv_heads;
-  const int u = blockIdx.y, t0 = blockIdx.x * kThreads, t = t0 + threadIdx.x;
-  const int r = (p.pool_kind == CKV_POOL_NONE) ? 0 : p.pool_size / 2;
-  const bool avg = p.pool_kind == CKV_POOL_AVG && r > 0;
-  const float pad = avg ? 0.f : -INFINITY;   // AVG counts outside positions as zeros, MAX ignores them
+  const int u = blockIdx.y, t0 = blockIdx.x * kSpan, tb = t0 + threadIdx.x * kPerThread;
   const float scale = (float)L / (float)s.window;
-  const float inv_size = 1.f / (float)p.pool_size;
+  const float inv_size = 1.f / (float)(2 * R + 1);
+  const float pad = AVG ? 0.f : -INFINITY;
   const float* hw = head_w + (int64_t)u * p.head_w_stride_unit;
-  float mass = 0.f, best = -INFINITY;
+  // a CTA whose staged range lies inside the prefix needs no range checks at all
+  const bool interior = t0 - kHalo >= 0 && t0 + kSpan + kHalo <= n;
+  float mass[kPerThread], best[kPerThread];
+#pragma unroll
+  for (int e = 0; e < kPerThread; ++e) mass[e] = 0.f, best[e] = -INFINITY;
   for (int h0 = 0; h0 < H; h0 += kHeadBatch) {
     const int nh = min(kHeadBatch, H - h0);
     __syncthreads();
-    for (int e = threadIdx.x; e < nh * (kThreads + 2 * r); e += kThreads) {
-      const int hh = e / (kThreads + 2 * r), i = e - hh * (kThreads + 2 * r);
-      const int tt = t0 - r + i;
-      const float* c = csum + ((int64_t)u * H + h0 + hh) * L;
-      // positions inside [0, L) are loaded as they are (the mass needs the window columns too);
-      // the pooling below replaces what lies outside the prefix by the pad value
-      tile[hh][i] = (tt >= 0 && tt < L) ? c[tt] : 0.f;
+    {
+      // all loads of the batch first, then the stores: the loads are independent and overlap
+      constexpr int kIters = (kWidth + kThreads - 1) / kThreads;
+      float buf[kHeadBatch][kIters];
+#pragma unroll
+      for (int hh = 0; hh < kHeadBatch; ++hh) {
+        const float* c = csum + ((int64_t)u * H + h0 + (hh < nh ? hh : 0)) * L;
+#pragma unroll
+        for (int it = 0; it < kIters; ++it) {
+          const int i = threadIdx.x + it * kThreads;
+          const int tt = t0 - kHalo + i;
+          buf[hh][it] = (hh < nh && i < kWidth && (interior || (tt >= 0 && tt < L))) ? c[tt] : 0.f;
+        }
+      }
+#pragma unroll
+      for (int hh = 0; hh < kHeadBatch; ++hh) {
+#pragma unroll
+        for (int it = 0; it < kIters; ++it) {
+          const int i = threadIdx.x + it * kThreads;
+          if (i < kWidth) tile[hh][i] = buf[hh][it];
+        }
+      }
     }
     __syncthreads();
     for (int hh = 0; hh < nh; ++hh) {
       const int h = h0 + hh;
-      const float* row = tile[hh] + threadIdx.x;   // row[i] = c_h[t - r + i]
-      if (t < L) mass += row[r];
-      if (t < n) {
-        float v;
-        if (avg) {
-          float acc = 0.f;
-          for (int i = 0; i <= 2 * r; ++i) {
-            const int tt = t - r + i;
-            acc += (tt >= 0 && tt < n) ? row[i] : pad;
-          }
-          v = acc * scale * inv_size;
-        } else {
-          float m = -INFINITY;
-          for (int i = 0; i <= 2 * r; ++i) {
-            const int tt = t - r + i;
-            m = fmaxf(m, (tt >= 0 && tt < n) ? row[i] : pad);
-          }
-          v = m * scale;
+      float win[kWin];   // win[i] = c_h[tb - kHalo + i]
+      const float4* src = reinterpret_cast<const float4*>(tile[hh] + threadIdx.x * kPerThread);
+#pragma unroll
+      for (int q4 = 0; q4 < kWin / 4; ++q4) {
+        const float4 x = src[q4];
+        win[4 * q4] = x.x, win[4 * q4 + 1] = x.y, win[4 * q4 + 2] = x.z, win[4 * q4 + 3] = x.w;
+      }
+#pragma unroll
+      for (int e = 0; e < kPerThread; ++e)
+        if (interior || tb + e < L) mass[e] += win[kHalo + e];
+      if (!interior) {   // the pooling only sees the prefix [0, n)
+#pragma unroll
+        for (int i = 0; i < kWin; ++i) {
+          const int tt = tb - kHalo + i;
+          if (tt < 0 || tt >= n) win[i] = pad;
         }
-        best = fmaxf(best, hw[h] * v);
+      }
+      const float w = hw[h];
+#pragma unroll
+      for (int e = 0; e < kPerThread; ++e) {
+        float v = win[kHalo + e - R];
+#pragma unroll
+        for (int i = 1; i <= 2 * R; ++i) v = AVG ? v + win[kHalo + e - R + i] : fmaxf(v, win[kHalo + e - R + i]);
+        v = AVG ? v * scale * inv_size : v * scale;
+        best[e] = fmaxf(best[e], w * v);
       }
       if ((h + 1) % G == 0) {  // last head of its KV group
-        if (t < n) scores[((int64_t)u * s.n_kv_heads + h / G) * n + t] = best;
-        best = -INFINITY;
+        float* out = scores + ((int64_t)u * s.n_kv_heads + h / G) * n;
+#pragma unroll
+        for (int e = 0; e < kPerThread; ++e) {
+          if (tb + e < n) out[tb + e] = best[e];
+          best[e] = -INFINITY;
+        }
       }
     }
   }
-  if (t < L) colmass[(int64_t)u * L + t] = mass;
+#pragma unroll
+  for (int e = 0; e < kPerThread; ++e)
+    if (tb + e < L) colmass[(int64_t)u * L + tb + e] = mass[e];
+}
+
+template <int R>
+void launch_r(bool avg, dim3 grid, cudaStream_t st, const ckv_shape& s, const ckv_params& p, const float* csum,
+              const float* head_w, float* scores, float* colmass) {
+  if (avg) pool_weight_max_mass<R, true><<<grid, kThreads, 0, st>>>(s, p, csum, head_w, scores, colmass);
+  else pool_weight_max_mass<R, false><<<grid, kThreads, 0, st>>>(s, p, csum, head_w, scores, colmass);
 }
 
 }  // namespace
 
 cudaError_t launch_epilogue(const ckv_shape& s, const ckv_params& p, const float* csum, const float* head_w,
                             float* scores, float* colmass, cudaStream_t st) {
-  dim3 grid((s.seq_len + kThreads - 1) / kThreads, s.n_units);
-  pool_weight_max_mass<<<grid, kThreads, 0, st>>>(s, p, csum, head_w, scores, colmass);
+  dim3 grid((s.seq_len + kSpan - 1) / kSpan, s.n_units);
+  const int r = (p.pool_kind == CKV_POOL_NONE) ? 0 : p.pool_size / 2;
+  const bool avg = p.pool_kind == CKV_POOL_AVG && r > 0;
+  switch (r) {
+    case 0: launch_r<0>(false, grid, st, s, p, csum, head_w, scores, colmass); break;
+    case 1: launch_r<1>(avg, grid, st, s, p, csum, head_w, scores, colmass); break;
+    case 2: launch_r<2>(avg, grid, st, s, p, csum, head_w, scores, colmass); break;
+    case 3: launch_r<3>(avg, grid, st, s, p, csum, head_w, scores, colmass); break;
+    case 4: launch_r<4>(avg, grid, st, s, p, csum, head_w, scores, colmass); break;
+    case 5: launch_r<5>(avg, grid, st, s, p, csum, head_w, scores, colmass); break;
+    case 6: launch_r<6>(avg, grid, st, s, p, csum, head_w, scores, colmass); break;
+    default: launch_r<7>(avg, grid, st, s, p, csum, head_w, scores, colmass); break;
+  }
   count_launch();
   return cudaGetLastError();
 }

@@ -8,21 +8,21 @@
 //   P2 (column sums)     D[key, row]  = K_tile . Q_blk^T   (the same shared-memory tiles, operands
 //        swapped): one TMEM lane per key, so c_h[t] = sum_i 2^(x[i,t] - bias_i) is thread-local.
 // A "chunk" is one (unit, KV head, block of 128 query rows); a "run" is a few consecutive key tiles of
-// a chunk.  CTA b takes P1 runs b, b+grid, ... and the P2 runs that trail them by a fixed lag, one tile
-// of each in turn, so the second read of a K tile comes from L2 while its chunk's statistics are
-// complete.  Warp roles:
-//   warp 0       producer (one thread): computes the schedule, issues the TMA loads and hands every
-//                sub-item (one tile of one pass) to the others through a descriptor ring in shared
-//                memory.  Sub-item j uses K stage j % 5 and TMEM buffer j % 4.  P1 tiles sit at even j,
-//                P2 tiles at odd j (a slot without work carries a no-op), and once P1 has ended P2
-//                takes both.  A P2 chunk whose statistics are not final yet never blocks P1: its slot
-//                carries a no-op and the tile is issued later.
+// a chunk.  CTAs take runs from two global queues (atomic counters), one per pass, in run order: P1
+// runs can always be taken; a P2 run can start once its chunk's statistics are final, which happens
+// shortly after the chunk's last P1 run, so the second read of a K tile usually comes from L2.  Results
+// do not depend on which CTA takes which run.  Warp roles:
+//   warp 0       producer (one thread): hands runs to two "lanes" (the even and the odd sub-items),
+//                issues the TMA loads and describes every sub-item (one tile of one pass) to the others
+//                through a descriptor ring in shared memory.  Sub-item j uses K stage j % 5, TMEM buffer
+//                j % 4 and the Q buffer of lane j % 2.  The odd lane prefers P2 runs and the even lane P1
+//                runs; a lane whose preferred queue has nothing ready takes a run of the other pass.
 //   warps 1, 19  MMA issuers (one thread each, even / odd j): tcgen05.mma M = N = K = 128 into one of four
 //                128-column TMEM buffers.
 //   warps 2..17  consumers: four groups, one per TMEM buffer, each with one warp per lane quadrant,
-//                read the accumulators back with tcgen05.ld.  Groups 0 and 2 see the P1 tiles.
-//   warp 18      scout: walks the CTA's P2 runs ahead of the producer, waits for a chunk's statistics
-//                and stages its 128 row biases in shared memory.
+//                read the accumulators back with tcgen05.ld.
+//   warp 18      scout: reserves the CTA's next P2 runs, waits for their chunks' statistics and stages
+//                their 128 row biases in shared memory.
 // K and Q tiles arrive by TMA (128-byte swizzle) and feed tcgen05.mma directly.
 //
 // Every wait is bounded: an mbarrier or flag wait that exceeds its time limit records a code in the
@@ -61,15 +61,14 @@ constexpr float kScale = 0.12751743074602467f;
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 
 // Tunables of the schedule (process-wide; see ckv_set_tunable).
-std::atomic<int> g_run_tiles{4};        // key tiles per run
-std::atomic<int> g_lag_slack_pct{200};  // extra lag of the P2 stream, in percent of the grid size
+std::atomic<int> g_run_tiles{8};        // key tiles per run
 std::atomic<int> g_l2_hints{1};         // 1: P1 loads keep their lines (evict_last), P2 loads release them
 
 struct TcArgs {
   int Nu, H, Hkv, G, L, W, n;
   int RB, hpb;          // row blocks per KV group; query heads per row block (128 / W)
   int T, run, RPC, C;   // key tiles per chunk; tiles per run; runs per chunk; chunks
-  int NR, DR;           // runs in total; lag of the P2 stream behind the P1 stream, in runs
+  int NR;               // runs in total
   int ppr, expected;    // partial pairs per run (1 or 2); pairs per (chunk, lane quadrant)
   int hints;
   uint32_t q_bytes;     // bytes of one Q block load
@@ -79,6 +78,7 @@ struct TcArgs {
   float2* stat;         // [C][128]          (row max, row max + log2 row sum)
   int* done;            // [C][4]
   int* ready;           // [C]
+  int* queue;           // [2] next P1 run and next P2 run to hand out
   int* status;
 };
 
@@ -234,32 +234,44 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
+// 2^x for x <= 0 on the FMA and integer pipes (the exponential unit is the scan's busiest pipe, so a
+// share of the exponentials goes here instead): x = n + f with n = round(x), f in [-0.5, 0.5];
+// 2^f by a degree-4 polynomial fitted for relative error (3e-6); 2^n by adding n to the exponent field.
+// Inputs below -125 are raised to -125 (2^-125 stands in for zero).
+__device__ __forceinline__ float ex2_poly(float x) {
+  x = fmaxf(x, -125.f);
+  const float t = x + 12582912.f;            // 1.5 * 2^23: the low mantissa bits of t hold n
+  const float f = x - (t - 12582912.f);
+  float p = fmaf(f, 9.582851277e-03f, 5.590642810e-02f);
+  p = fmaf(f, p, 2.402409867e-01f);
+  p = fmaf(f, p, 6.931241930e-01f);
+  p = fmaf(f, p, 1.f);
+  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
+// Which of the 32 values of a TMEM slice take the polynomial instead of the exponential unit.
+__device__ __forceinline__ constexpr bool use_poly(int jj) { return (jj & 3) == 3; }
+
 __device__ __forceinline__ int ld_acquire(const int* p) {
   int v;
   asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
 
-// One of a CTA's two streams of runs: run m of the stream is global run blockIdx.x + m * gridDim.x - shift.
-struct RunStream {
-  int m, k, tr, chunk, ric, u, g, head0, heads;
-  bool done;
-  __device__ void init() { m = 0, k = 0, tr = 0, chunk = -1, ric = 0, u = 0, g = 0, head0 = 0, heads = 1, done = false; }
-  // Moves to run m (or the next one that exists) and works out where its chunk lives.
-  __device__ void next_run(const TcArgs& a, int shift) {
-    int rho;
-    for (;; ++m) {
-      rho = (int)blockIdx.x + m * (int)gridDim.x - shift;
-      if (rho >= a.NR) {
-        done = true, tr = 0;
-        return;
-      }
-      if (rho >= 0) break;
-    }
+// What one of the two slot lanes (even / odd sub-items) is working on: a run of either pass, and the
+// state of the lane's Q buffer.
+struct Lane {
+  int type, k, tr, chunk, ric, u, g, head0, heads, gen;   // the run in hand (k == tr: none)
+  int q_chunk, q_last, q_loads;  // chunk whose rows the lane's Q buffer holds; its last reader; loads so far
+  __device__ void init() {
+    type = kNop, k = 0, tr = 0, chunk = -1, ric = 0, u = 0, g = 0, head0 = 0, heads = 1, gen = 0;
+    q_chunk = -1, q_last = -1000, q_loads = 0;
+  }
+  // Takes global run rho of pass ty and works out where its chunk lives.
+  __device__ void take(const TcArgs& a, int rho, int ty, int generation) {
+    type = ty, k = 0, gen = generation;
     const int c = rho / a.RPC;
     ric = rho - c * a.RPC;
     tr = min(a.run, a.T - ric * a.run);
-    k = 0;
     if (c != chunk) {
       chunk = c;
       const int per_unit = a.Hkv * a.RB;
@@ -276,19 +288,21 @@ struct RunStream {
 // ------------------------------------------------------------------------------------ shared memory
 struct __align__(1024) Smem {
   uint8_t k[kStages][kTileBytes];  // K tiles: two 64-column halves of [128 rows][128 bytes], swizzled
-  uint8_t q[2][kTileBytes];        // query rows of the P1 stream's chunk and of the P2 stream's chunk
-  float nbias[kBiasBufs][kTile];   // negated row biases -(max + log2 sum) of the P2 stream's recent chunks
+  uint8_t q[2][kTileBytes];        // query rows of the run on the even lane and of the run on the odd lane
+  float nbias[kBiasBufs][kTile];   // negated row biases -(max + log2 sum) of the most recent P2 runs
   Desc desc[kRing];
   // full[j % kFullBars] says sub-item j's K tile has landed.  There are two barriers per K stage so that
   // each of the two MMA threads (even / odd j) sees every phase of the barriers it waits on: a parity wait
   // is only sound for a waiter that never skips a phase.
   uint64_t full[kFullBars], empty[kStages], tmem_full[kTmemBufs], tmem_empty[kTmemBufs];
-  uint64_t q_full[2];              // a stream's Q rows have landed (both MMA threads wait on it)
+  uint64_t q_full[2];              // a lane's Q rows have landed
   uint32_t tmem_base;
   int abort_flag;
-  int p2_ready_gen;   // scout -> producer: biases of P2 chunk generations up to this one are staged
-  int gen_started;    // producer -> scout: latest P2 chunk generation whose first tile was issued ...
-  int gen_start_j[kBiasBufs];  // ... and the sub-item index of that first tile, per generation % kBiasBufs
+  int p2_ready_gen;   // scout -> producer: P2 runs ("generations", counted from 1) up to this one are staged ...
+  int p2_rho[kBiasBufs];       // ... which global run each of them is, per generation % kBiasBufs ...
+  int p2_total;       // ... and how many there will be in all (-1 until the scout knows)
+  int gen_fin[kBiasBufs];      // producer -> scout: generation whose last tile was issued, per generation % kBiasBufs ...
+  int gen_last_j[kBiasBufs];   // ... and the sub-item index of that last tile
   int prod_j;         // producer -> scout: index of the sub-item being issued
 };
 static_assert(sizeof(Smem) <= 232448, "shared memory of one CTA");
@@ -371,7 +385,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     mbar_init(smem_u32(&sm.q_full[1]), 1);
     sm.abort_flag = 0;
     sm.p2_ready_gen = 0;
-    sm.gen_started = 0;
+    sm.p2_total = -1;
+    for (int e = 0; e < kBiasBufs; ++e) sm.gen_fin[e] = 0, sm.gen_last_j[e] = 0, sm.p2_rho[e] = 0;
     sm.prod_j = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -384,111 +399,115 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = sm.tmem_base;
+  const int NR = a.NR;
+  int* const queue = a.queue;
 
   if (warp == 0) {
     // ================================================================= producer: schedule + TMA (one thread)
     if (lane == 0) {
-      RunStream st0, st1;  // the P1 stream and the P2 stream
-      st0.init(), st1.init();
-      st0.next_run(a, 0), st1.next_run(a, a.DR);
-      int q_chunk0 = -1, q_chunk1 = -1;      // chunk whose rows each stream's Q buffer holds
-      // last even and last odd sub-item that read each stream's Q buffer (one per MMA thread)
-      int q_last0e = -1000, q_last0o = -1000, q_last1e = -1000, q_last1o = -1000;
-      int q_loads0 = 0, q_loads1 = 0;        // loads into each stream's Q buffer so far
-      int gen = 0;  // P2 chunks entered so far; biases of generation e live in nbias[e % kBiasBufs]
+      Lane ln0, ln1;       // even and odd sub-items
+      ln0.init(), ln1.init();
+      int gen = 0;         // P2 runs started so far; the biases of run e live in nbias[e % kBiasBufs]
+      int p1_next = atomicAdd(queue, 1);   // the CTA's next P1 run, fetched one run ahead
       const uint64_t pol_q = policy_evict_last();
       const uint64_t pol_k0 = a.hints ? policy_evict_last() : policy_evict_normal();
       const uint64_t pol_k1 = a.hints ? policy_evict_first() : policy_evict_normal();
       bool ok = true;
       int j = 0;
-      // Issues the next tile of a stream as sub-item j (ty is a compile-time constant at both call sites).
-      auto issue = [&](RunStream& r, const int ty, int& q_chunk, int& q_last_e, int& q_last_o, int& q_loads,
-                       const uint64_t pol_k) {
+      unsigned long long t_busy = global_ns();   // when the producer last had a tile to issue
+      auto p2_done = [&] { return gen == *(volatile int*)&sm.p2_total; };
+      // Hands the lane its next run.  The even lane prefers P1 and the odd lane P2, so that in the steady
+      // state the two passes alternate; a lane whose preferred queue has nothing to give (no P2 run whose
+      // chunk is final, or no P1 run left) takes a run of the other pass instead of idling.
+      auto refill = [&](Lane& ln, const bool prefer_p2) {
+        const bool p2_ok = *(volatile int*)&sm.p2_ready_gen >= gen + 1;   // the scout has staged the next P2 run
+        const bool p1_ok = p1_next < NR;
+        if (p2_ok && (prefer_p2 || !p1_ok)) {
+          __threadfence_block();
+          ++gen;
+          ln.take(a, *(volatile int*)&sm.p2_rho[gen % kBiasBufs], kP2, gen);
+        } else if (p1_ok) {
+          ln.take(a, p1_next, kP1, 0);
+          p1_next = atomicAdd(queue, 1);
+        }
+      };
+      // Issues the next tile of the lane's run as sub-item j.
+      auto issue = [&](Lane& ln, const int lane_id) {
         const int stage = j % kStages;
         const uint32_t bar = smem_u32(&sm.full[j % kFullBars]);
         int4* d = reinterpret_cast<int4*>(&sm.desc[j % kRing]);
-        const bool reload = r.chunk != q_chunk;
+        const bool reload = ln.chunk != ln.q_chunk;
         if (reload) {
-          // The MMAs that read the stream's old rows must have completed, those of either MMA thread (the
-          // two complete independently, and a thread still waiting for the old rows' barrier phase must not
-          // be overtaken by the next load).  The wait on this sub-item's K stage covers sub-items up to
+          // The MMAs that read the lane's old rows must have completed (they all come from the lane's own
+          // MMA thread, in order).  The wait on this sub-item's K stage covers sub-items up to
           // j - kStages; a younger reader needs its own stage's barrier.
-          if (q_last_e > j - kStages)
-            ok = mbar_wait(smem_u32(&sm.empty[q_last_e % kStages]), (q_last_e / kStages) & 1, abort_flag, a.status,
-                           12 | (j << 8));
-          if (ok && q_last_o > j - kStages)
-            ok = mbar_wait(smem_u32(&sm.empty[q_last_o % kStages]), (q_last_o / kStages) & 1, abort_flag, a.status,
+          if (ln.q_last > j - kStages)
+            ok = mbar_wait(smem_u32(&sm.empty[ln.q_last % kStages]), (ln.q_last / kStages) & 1, abort_flag, a.status,
                            12 | (j << 8));
           if (!ok) return;
-          ++q_loads;
-          q_chunk = r.chunk;
-          if (ty == kP2) {
-            ++gen;
-            *(volatile int*)&sm.gen_start_j[gen % kBiasBufs] = j;
-            __threadfence_block();
-            *(volatile int*)&sm.gen_started = gen;
-          }
+          ++ln.q_loads;
+          ln.q_chunk = ln.chunk;
         }
-        if (j & 1) q_last_o = j;
-        else q_last_e = j;
-        const int tile = r.ric * a.run + r.k;
-        // the n-th load of a stream's rows (n = 0, 1, ...) completes phase n of its barrier: wait for parity n & 1
-        const int q_phase = (q_loads - 1) & 1;
-        d[0] = make_int4(ty | (q_phase << 9), r.chunk, tile, (r.k + 2 >= r.tr) ? r.ric * a.ppr + (r.k & 1) : -1);
-        d[1] = make_int4(r.k < 2, r.u * a.H + r.head0, r.heads, gen % kBiasBufs);
+        ln.q_last = j;
+        const int tile = ln.ric * a.run + ln.k;
+        // the n-th load of a lane's rows (n = 0, 1, ...) completes phase n of its barrier: wait for parity n & 1
+        const int q_phase = (ln.q_loads - 1) & 1;
+        d[0] = make_int4(ln.type | (q_phase << 9), ln.chunk, tile,
+                         (ln.k + 2 >= ln.tr) ? ln.ric * a.ppr + (ln.k & 1) : -1);
+        d[1] = make_int4(ln.k < 2, ln.u * a.H + ln.head0, ln.heads, ln.gen % kBiasBufs);
         mbar_arrive_expect_tx(bar, kTileBytes);
         if (reload) {
-          const uint32_t qbar = smem_u32(&sm.q_full[ty]);
+          const uint32_t qbar = smem_u32(&sm.q_full[lane_id]);
           mbar_arrive_expect_tx(qbar, a.q_bytes);
-          tma_load_5d(&q_map, smem_u32(sm.q[ty]), qbar, 0, 0, r.head0, 0, r.u, pol_q);
-          if (a.q_split) tma_load_5d(&q_map, smem_u32(sm.q[ty]) + kHalfBytes, qbar, 0, 0, r.head0, 1, r.u, pol_q);
+          tma_load_5d(&q_map, smem_u32(sm.q[lane_id]), qbar, 0, 0, ln.head0, 0, ln.u, pol_q);
+          if (a.q_split)
+            tma_load_5d(&q_map, smem_u32(sm.q[lane_id]) + kHalfBytes, qbar, 0, 0, ln.head0, 1, ln.u, pol_q);
         }
-        tma_load_5d(&k_map, smem_u32(sm.k[stage]), bar, 0, tile * kTile, 0, r.g, r.u, pol_k);
+        tma_load_5d(&k_map, smem_u32(sm.k[stage]), bar, 0, tile * kTile, 0, ln.g, ln.u,
+                    ln.type == kP1 ? pol_k0 : pol_k1);
         TC_TRACE(1, j);
-        if (++r.k == r.tr) {
-          ++r.m;
-          r.next_run(a, ty == kP1 ? 0 : a.DR);
+        if (++ln.k == ln.tr && ln.type == kP2) {
+          // the run's biases may be replaced once its readers are done: tell the scout where it ended
+          *(volatile int*)&sm.gen_last_j[ln.gen % kBiasBufs] = j;
+          __threadfence_block();
+          *(volatile int*)&sm.gen_fin[ln.gen % kBiasBufs] = ln.gen;
         }
       };
-      while (ok && !(st0.done && st1.done)) {
+      while (ok) {
+        if (ln0.k == ln0.tr && ln1.k == ln1.tr && p1_next >= NR && p2_done()) break;
+        int idle = 0;
 #pragma unroll
         for (int slot = 0; slot < 2; ++slot, ++j) {
-          // Even slots carry the P1 stream while it lasts; P2 tiles take the odd slots, never ahead of
-          // the P1 tile they are paired with, and both slots once P1 has ended.
-          int ty = kNop;
-          if (slot == 0 && !st0.done) {
-            ty = kP1;
-          } else if (!st1.done && (st0.done || st1.m < st0.m || (st1.m == st0.m && st1.k < st0.k))) {
-            ty = kP2;
-            if (st1.k == 0 && st1.chunk != q_chunk1) {
-              // a new chunk: its biases must have been staged by the scout warp
-              if (*(volatile int*)&sm.p2_ready_gen < gen + 1) {
-                ty = kNop;
-                TC_COUNT(3);
-                if (st0.done) __nanosleep(100);
-                if (*abort_flag) ok = false;
-              } else {
-                __threadfence_block();
-              }
-            }
-          }
+          Lane& ln = slot == 0 ? ln0 : ln1;
+          if (ln.k == ln.tr) refill(ln, slot == 1);
           ok = ok && mbar_wait(smem_u32(&sm.empty[j % kStages]), ((j / kStages) & 1) ^ 1, abort_flag, a.status,
                                11 | (j << 8));
           TC_TRACE(0, j);
           if (!ok) break;
           TC_COUNT(0);
-          if (ty == kNop && !st1.done) TC_COUNT(4);
-          if (ty != kNop) TC_COUNT(1 + ty);
           *(volatile int*)&sm.prod_j = j;
-          if (ty == kP1) {
-            issue(st0, kP1, q_chunk0, q_last0e, q_last0o, q_loads0, pol_k0);
-          } else if (ty == kP2) {
-            issue(st1, kP2, q_chunk1, q_last1e, q_last1o, q_loads1, pol_k1);
+          if (ln.k < ln.tr) {
+            TC_COUNT(1 + ln.type);
+            issue(ln, slot);
           } else {
+            TC_COUNT(3);
+            ++idle;
             sm.desc[j % kRing].type = kNop;
             mbar_arrive(smem_u32(&sm.full[j % kFullBars]));
           }
           if (!ok) break;
+        }
+        if (idle == 2) {  // nothing to issue on either lane: P2 runs are waiting for their chunks
+          __nanosleep(200);
+          if (*abort_flag) {
+            ok = false;
+          } else if (global_ns() - t_busy > kWaitLimitNs) {
+            *abort_flag = 1;
+            atomicCAS(a.status, 0, 16 | (j << 8));
+            ok = false;
+          }
+        } else {
+          t_busy = global_ns();
         }
       }
       // one stop marker per consumer group
@@ -505,47 +524,76 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       }
     }
   } else if (warp == kScoutWarp) {
-    // ================================================================= scout: stages the biases of the P2 chunks
-    int gen = 0, prev_chunk = -1;
+    // ================================================================= scout: stages the biases of the P2 runs
+    // Reserves P2 runs from the global queue, a window of kBiasBufs at a time (lane i looks after the run
+    // that will be this CTA's generation G + i), polls the readiness flags of their chunks together, and
+    // stages them in order: copies the negated biases into shared memory and tells the producer which
+    // run it is.
+    unsigned long long t_progress = global_ns();
     bool ok = true;
-    for (int m = 0; ok; ++m) {
-      const int rho = (int)blockIdx.x + m * (int)gridDim.x - a.DR;
-      if (rho >= a.NR) break;
-      if (rho < 0) continue;
-      const int c = rho / a.RPC;
-      if (c == prev_chunk) continue;
-      prev_chunk = c;
-      ++gen;
-      if (lane == 0) {
-        // nbias[gen % kBiasBufs] last served generation gen - kBiasBufs, whose tiles all precede the first
-        // tile of generation gen - kBiasBufs + 1; a tile's readers are done once the producer has got
-        // kStages + kTmemBufs sub-items past it (it waits for the K stage of sub-item j - kStages to be free,
-        // whose MMA waited for the TMEM buffer of sub-item j - kStages - kTmemBufs).
-        if (gen > kBiasBufs) {
-          const int g1 = gen - kBiasBufs + 1;
-          ok = wait_flag(
-              [&] {
-                if (*(volatile int*)&sm.gen_started < g1) return false;
-                __threadfence_block();
-                return *(volatile int*)&sm.prod_j >=
-                       *(volatile int*)&sm.gen_start_j[g1 % kBiasBufs] + kStages + kTmemBufs - 1;
-              },
-              200, abort_flag, a.status, 15);
+    int G = 1;          // next generation to stage
+    // run reserved for generation G + lane: the first window in one step, so that it is in increasing order
+    // (later reservations are made one at a time and the counter only grows)
+    int my_rho = 0;
+    if (lane == 0) my_rho = atomicAdd(queue + 1, kBiasBufs);
+    my_rho = __shfl_sync(0xffffffffu, my_rho, 0) + lane;   // every lane takes part in the shuffle
+    if (lane >= kBiasBufs) my_rho = NR;
+    bool mine = false;  // its chunk is known to be final
+    int it = 0;
+    while (ok) {
+      const int rho0 = __shfl_sync(0xffffffffu, my_rho, 0);
+      if (rho0 >= NR) break;   // the queue is exhausted (runs are handed out in increasing order)
+      if (!mine && my_rho < NR) mine = ld_acquire(a.ready + my_rho / a.RPC) >= 4;
+      const unsigned ready_mask = __ballot_sync(0xffffffffu, mine);
+      bool staged = false;
+      if (ready_mask & 1u) {
+        // nbias[G % kBiasBufs] last served run G - kBiasBufs: all of its tiles must have been issued, and a
+        // tile's readers are done once the producer has got kStages + kTmemBufs sub-items past it (it waits
+        // for the K stage of sub-item j - kStages to be free, whose MMA waited for the TMEM buffer of
+        // sub-item j - kStages - kTmemBufs).
+        bool free_buf = true;
+        if (G > kBiasBufs) {
+          free_buf = *(volatile int*)&sm.gen_fin[G % kBiasBufs] == G - kBiasBufs;
+          if (free_buf) {
+            __threadfence_block();
+            free_buf = *(volatile int*)&sm.prod_j >= *(volatile int*)&sm.gen_last_j[G % kBiasBufs] + kStages + kTmemBufs;
+          }
         }
-        // the chunk's row statistics must be final
-        ok = ok && wait_flag([&] { return ld_acquire(a.ready + c) >= 4; }, 100, abort_flag, a.status, 13);
+        free_buf = __shfl_sync(0xffffffffu, free_buf ? 1 : 0, 0) != 0;
+        if (free_buf) {
+          const float2* stp = a.stat + (int64_t)(rho0 / a.RPC) * kTile + 4 * lane;
+          const float2 s0 = __ldcg(stp), s1 = __ldcg(stp + 1), s2 = __ldcg(stp + 2), s3 = __ldcg(stp + 3);
+          reinterpret_cast<float4*>(sm.nbias[G % kBiasBufs])[lane] = make_float4(-s0.y, -s1.y, -s2.y, -s3.y);
+          if (lane == 0) *(volatile int*)&sm.p2_rho[G % kBiasBufs] = rho0;
+          __syncwarp();
+          if (lane == 0) {
+            __threadfence_block();
+            *(volatile int*)&sm.p2_ready_gen = G;
+          }
+          ++G;
+          // shift the window down by one and reserve a run for its new last place
+          const int nrho = __shfl_down_sync(0xffffffffu, my_rho, 1);
+          const bool nmine = __shfl_down_sync(0xffffffffu, mine ? 1 : 0, 1) != 0;
+          my_rho = nrho, mine = nmine;
+          if (lane == kBiasBufs - 1) my_rho = atomicAdd(queue + 1, 1), mine = false;
+          if (lane >= kBiasBufs) my_rho = NR, mine = false;
+          staged = true;
+          t_progress = global_ns();
+        }
       }
-      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-      if (!ok) break;
-      const float2* stp = a.stat + (int64_t)c * kTile + 4 * lane;
-      const float2 s0 = __ldcg(stp), s1 = __ldcg(stp + 1), s2 = __ldcg(stp + 2), s3 = __ldcg(stp + 3);
-      reinterpret_cast<float4*>(sm.nbias[gen % kBiasBufs])[lane] = make_float4(-s0.y, -s1.y, -s2.y, -s3.y);
-      __syncwarp();
-      if (lane == 0) {
-        __threadfence_block();
-        *(volatile int*)&sm.p2_ready_gen = gen;
+      if (!staged) {
+        __nanosleep(100);
+        if ((++it & 63) == 0) {
+          bool give_up = *abort_flag != 0;
+          if (!give_up && global_ns() - t_progress > kWaitLimitNs) {
+            give_up = true;
+            if (lane == 0) *abort_flag = 1, atomicCAS(a.status, 0, 13 | (G << 8));
+          }
+          ok = !__any_sync(0xffffffffu, give_up);
+        }
       }
     }
+    if (lane == 0) *(volatile int*)&sm.p2_total = G - 1;   // every reserved run that exists has been staged
   } else if (warp == 1 || warp == kMma2Warp) {
     // ================================================================= MMA issuers
     // Two threads take turns (even / odd sub-items), so that one waits and sets up while the other's
@@ -564,11 +612,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         ok = mbar_wait(smem_u32(&sm.tmem_empty[buf]), ((j / kTmemBufs) & 1) ^ 1, abort_flag, a.status, 22 | (j << 8));
         if (!ok) break;
         if (type == kP1 || type == kP2) {
-          ok = mbar_wait(smem_u32(&sm.q_full[type]), (tq >> 9) & 1, abort_flag, a.status, 23 | (j << 8));
+          ok = mbar_wait(smem_u32(&sm.q_full[j & 1]), (tq >> 9) & 1, abort_flag, a.status, 23 | (j << 8));
           if (!ok) break;
           tc_fence_after();
           const uint32_t kd = k_lo + stage * (kTileBytes >> 4);
-          const uint32_t qd = q_lo + type * (kTileBytes >> 4);
+          const uint32_t qd = q_lo + (j & 1) * (kTileBytes >> 4);
           const uint32_t a_lo = type == kP1 ? qd : kd, b_lo = type == kP1 ? kd : qd;
           const uint32_t d = tmem_base + buf * kTile;
 #pragma unroll
@@ -614,17 +662,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         // ---------------------------------------------------------- P1: running (max, sum) of this row
         if (d.first) m_run = kMinRowMax, l_run = 0.f;
         const int limit = a.n + row % W;   // last key this window row sees
-        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll 1
-        for (int cc = 0; cc < 4; ++cc) {
-          float v[32];
-          load_logits(taddr + cc * 32, v, tail, t0 + cc * 32, limit);
-#pragma unroll
-          for (int jj = 0; jj < 32; ++jj) mx[jj & 3] = fmaxf(mx[jj & 3], v[jj]);
-        }
-        const float m_new = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * kScale, m_run);
-        const float negm = -m_new;
-        float sum[4] = {l_run * ex2(m_run - m_new), 0.f, 0.f, 0.f};
 #pragma unroll 1
         for (int cc = 0; cc < 4; ++cc) {
           float v[32];
@@ -634,11 +671,20 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_empty);
           }
+          float mx[4] = {v[0], v[1], v[2], v[3]};
 #pragma unroll
-          for (int jj = 0; jj < 32; ++jj) sum[jj & 3] += ex2(fmaf(v[jj], kScale, negm));
+          for (int jj = 4; jj < 32; ++jj) mx[jj & 3] = fmaxf(mx[jj & 3], v[jj]);
+          const float m_new = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * kScale, m_run);
+          const float negm = -m_new;
+          float sum[4] = {l_run * ex2(m_run - m_new), 0.f, 0.f, 0.f};
+#pragma unroll
+          for (int jj = 0; jj < 32; ++jj) {
+            const float x = fmaf(v[jj], kScale, negm);
+            sum[jj & 3] += use_poly(jj) ? ex2_poly(x) : ex2(x);
+          }
+          l_run = (sum[0] + sum[1]) + (sum[2] + sum[3]);
+          m_run = m_new;
         }
-        l_run = (sum[0] + sum[1]) + (sum[2] + sum[3]);
-        m_run = m_new;
         if (d.part_slot >= 0) {
           // this group's last tile of the run: publish the pair; the last warp of the chunk's
           // quadrant merges all of them in slot order
@@ -678,7 +724,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
               const int jj = j4 * 4 + e;
-              float p = ex2(fmaf(v[jj], kScale, bb[e]));
+              const float x = fmaf(v[jj], kScale, bb[e]);
+              float p = use_poly(jj) ? ex2_poly(x) : ex2(x);
               if (tail) {
                 const int i = (cc * 32 + jj) % W;
                 if (t > a.n + i) p = 0.f;
@@ -800,14 +847,13 @@ TcLayout tc_layout(const ckv_shape& s) {
   t.C = (int64_t)s.n_units * s.n_kv_heads * t.RB;
   t.part_bytes = (size_t)t.C * (t.T + 2) * kTile * sizeof(float2);  // at most T + 1 pairs per chunk
   t.stat_bytes = (size_t)t.C * kTile * sizeof(float2);
-  t.flag_bytes = (size_t)t.C * 5 * sizeof(int);
+  t.flag_bytes = ((size_t)t.C * 5 + 2) * sizeof(int);
   return t;
 }
 
 int set_tc_tunable(const char* name, int value) {
   const std::string n(name);
   if (n == "run_tiles" && value >= 1 && value <= 64) return g_run_tiles.exchange(value);
-  if (n == "lag_slack_pct" && value >= 0 && value <= 1000) return g_lag_slack_pct.exchange(value);
   if (n == "l2_hints" && (value == 0 || value == 1)) return g_l2_hints.exchange(value);
   return -1;
 }
@@ -827,7 +873,6 @@ cudaError_t launch_score_tc(const ckv_shape& s, const void* q, const void* k, fl
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int grid = sms < a.NR ? sms : a.NR;
-  a.DR = a.RPC + (int)(((int64_t)grid * g_lag_slack_pct.load() + 99) / 100);
   const int t_last = a.T - (a.RPC - 1) * a.run;
   a.ppr = a.run < 2 ? 1 : 2;
   a.expected = (a.RPC - 1) * a.ppr + (t_last < 2 ? t_last : 2);
@@ -836,7 +881,7 @@ cudaError_t launch_score_tc(const ckv_shape& s, const void* q, const void* k, fl
   a.q_bytes = 2u * 64u * 2u * (uint32_t)a.W * (uint32_t)hpb_box;
   a.q_split = hpb_box * a.W < kTile;  // a short box would pack its halves closer than the operand layout wants
   a.csum = csum, a.part = (float2*)part, a.stat = (float2*)stat;
-  a.done = flags, a.ready = flags + 4 * a.C, a.status = status;
+  a.done = flags, a.ready = flags + 4 * a.C, a.queue = flags + 5 * a.C, a.status = status;
   CUtensorMap qm, km;
   {
     // Q: [unit][half][head][row][64]; box = one row block (hpb heads x W rows) x both halves

@@ -25,7 +25,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(ckv_shape s, const flo
                                                           const int32_t* __restrict__ offsets,
                                                           int32_t* __restrict__ indices) {
   __shared__ int whist[kWarps][256];   // one histogram per warp: no contention between warps
-  __shared__ int suffix[256];
+  __shared__ int totals[256];
   __shared__ uint32_t sh_prefix;
   __shared__ int sh_want;
   __shared__ int warp_gt[kWarps], warp_eq[kWarps];
@@ -91,25 +91,34 @@ __global__ void __launch_bounds__(kThreads) select_kernel(ckv_shape s, const flo
     }
     if (run_cnt) atomicAdd(&whist[warp][run_bin], run_cnt);
     __syncthreads();
+    // 256 threads add the per-warp histograms, then warp 0 (lane i owns digits 8 i .. 8 i + 7) finds the
+    // digit d with count(digit > d) < want <= count(digit >= d)
     if (threadIdx.x < 256) {
       int tot = 0;
 #pragma unroll 8
       for (int w = 0; w < kWarps; ++w) tot += whist[w][threadIdx.x];
-      suffix[threadIdx.x] = tot;
+      totals[threadIdx.x] = tot;
     }
     __syncthreads();
-    // suffix[b] = number of matching keys whose digit is >= b
-    for (int o = 1; o < 256; o <<= 1) {
-      int add = 0;
-      if (threadIdx.x < 256 && threadIdx.x + o < 256) add = suffix[threadIdx.x + o];
-      __syncthreads();
-      if (threadIdx.x < 256) suffix[threadIdx.x] += add;
-      __syncthreads();
-    }
-    if (threadIdx.x < 256) {
-      const int here = suffix[threadIdx.x], above = threadIdx.x < 255 ? suffix[threadIdx.x + 1] : 0;
-      if (here >= want && above < want) {   // exactly one digit qualifies
-        sh_prefix = prefix | ((uint32_t)threadIdx.x << shift);
+    if (warp == 0) {
+      int cnt[8], mine = 0;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) cnt[e] = totals[8 * lane + e], mine += cnt[e];
+      // above = number of matching keys in the digits of higher lanes
+      int incl = mine;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int x = __shfl_down_sync(0xffffffffu, incl, o);
+        if (lane + o < 32) incl += x;
+      }
+      int above = incl - mine;
+      if (above < want && incl >= want) {   // the digit lies in this lane's range: exactly one lane
+        int dgt = 7;
+        for (; dgt > 0; --dgt) {
+          if (above + cnt[dgt] >= want) break;
+          above += cnt[dgt];
+        }
+        sh_prefix = prefix | ((uint32_t)(8 * lane + dgt) << shift);
         sh_want = want - above;
       }
     }
