@@ -1,9 +1,13 @@
-// Per-head exact Top-k (Eq. 8's Top-B branch): a most-significant-digit radix select finds the
-// key of the k-th largest score, then one ordered compaction writes the kept positions in
-// ascending order; equal scores are resolved toward the lowest index, and the observation window
-// is appended.  One CTA per (unit, KV head); integer work only, bit-exact and deterministic.
-// Thread i owns the contiguous positions [i*chunk, (i+1)*chunk); when a head's prefix fits
-// (chunk <= 32) the keys stay in registers for all four digit passes and the compaction.
+// Per-head exact Top-k (Eq. 8's Top-B branch): a most-significant-bit-first search finds the key of
+// the k-th largest score, then one ordered compaction writes the kept positions in ascending order;
+// equal scores are resolved toward the lowest index, and the observation window is appended.
+// One CTA per (unit, KV head); integer work only, bit-exact and deterministic.
+// Warp w owns the contiguous positions [w * 32 * chunk, (w + 1) * 32 * chunk) and lane l of it the
+// positions w * 32 * chunk + 32 j + l, so that every load is coalesced and a ballot per j gives the
+// order inside the warp's range.  When a head's prefix fits (chunk <= 32) the keys stay in registers
+// and the search takes one bit per step: count the keys at or above the candidate (a compare per key,
+// one warp reduction, one barrier).  Longer prefixes use 8-bit digits with per-warp histograms and
+// re-read the scores in every pass.
 #include "ckv_common.cuh"
 
 namespace ckv {
@@ -24,8 +28,9 @@ __global__ void __launch_bounds__(kThreads) select_kernel(ckv_shape s, const flo
                                                           const int32_t* __restrict__ budgets,
                                                           const int32_t* __restrict__ offsets,
                                                           int32_t* __restrict__ indices) {
-  __shared__ int whist[kWarps][256];   // one histogram per warp: no contention between warps
+  __shared__ int whist[kCached ? 1 : kWarps][256];   // 8-bit path: one histogram per warp
   __shared__ int totals[256];
+  __shared__ int wcnt[2][kWarps];
   __shared__ uint32_t sh_prefix;
   __shared__ int sh_want;
   __shared__ int warp_gt[kWarps], warp_eq[kWarps];
@@ -44,39 +49,48 @@ __global__ void __launch_bounds__(kThreads) select_kernel(ckv_shape s, const flo
     return;
   }
 
-  const int chunk = (n + kThreads - 1) / kThreads;
-  const int t0 = min(threadIdx.x * chunk, n), t1 = min(t0 + chunk, n);
+  const int chunk = (n + kThreads - 1) / kThreads;      // positions per thread
+  const int base = warp * 32 * chunk + lane;            // position of (j = 0); (j) is base + 32 j
+  const int wend = min((warp + 1) * 32 * chunk, n);     // end of the warp's range
   uint32_t keys[kCached ? kCache : 1];
   if (kCached) {
 #pragma unroll
-    for (int j = 0; j < kCache; ++j) keys[j] = (t0 + j < t1) ? key_of(sc[t0 + j]) : 0u;
+    for (int j = 0; j < kCache; ++j) {
+      const int t = base + 32 * j;
+      keys[j] = (j < chunk && t < wend) ? key_of(sc[t]) : 0u;   // key 0 is below every real key
+    }
   }
 
-  // radix select, 8 bits per pass from the top: after the loop `prefix` is the key of the e-th
-  // largest score and `want` the number of scores equal to it that are kept
-  uint32_t prefix = 0, mask = 0;
+  uint32_t prefix = 0;
   int want = e;
-  for (int shift = 24; shift >= 0; shift -= 8) {
-    for (int i = lane; i < 256; i += 32) whist[warp][i] = 0;
-    __syncwarp();
-    // consecutive equal digits of a thread are added in one go (scores of one head share their top bits)
-    int run_bin = -1, run_cnt = 0;
+  if (kCached) {
+    // one bit per step: the k-th largest key is the largest value v with #{keys >= v} >= k
+    for (int bit = 31; bit >= 0; --bit) {
+      const uint32_t cand = prefix | (1u << bit);
+      int c[4] = {0, 0, 0, 0};
 #pragma unroll
-    for (int j = 0; j < (kCached ? kCache : 1); ++j) {
-      if (kCached) {
-        if (t0 + j < t1 && (keys[j] & mask) == prefix) {
-          const int bin = (keys[j] >> shift) & 0xff;
-          if (bin == run_bin) {
-            ++run_cnt;
-          } else {
-            if (run_cnt) atomicAdd(&whist[warp][run_bin], run_cnt);
-            run_bin = bin, run_cnt = 1;
-          }
-        }
+      for (int j = 0; j < kCache; ++j) c[j & 3] += keys[j] >= cand;
+      const int cw = __reduce_add_sync(0xffffffffu, (c[0] + c[1]) + (c[2] + c[3]));
+      if (lane == 0) wcnt[0][warp] = cw;
+      __syncthreads();
+      if (warp == 0) {
+        const int tot = __reduce_add_sync(0xffffffffu, wcnt[0][lane]);
+        if (lane == 0) wcnt[1][0] = tot;
       }
+      __syncthreads();
+      if (wcnt[1][0] >= e) prefix = cand;
     }
-    if (!kCached) {
-      for (int t = t0; t < t1; ++t) {
+  } else {
+    // 8 bits per pass from the top: after the loop `prefix` is the key of the e-th largest score
+    uint32_t mask = 0;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+      for (int i = lane; i < 256; i += 32) whist[warp][i] = 0;
+      __syncwarp();
+      // consecutive equal digits of a thread are added in one go (scores of one head share their top bits)
+      int run_bin = -1, run_cnt = 0;
+      for (int j = 0; j < chunk; ++j) {
+        const int t = base + 32 * j;
+        if (t >= wend) break;
         const uint32_t key = key_of(sc[t]);
         if ((key & mask) == prefix) {
           const int bin = (key >> shift) & 0xff;
@@ -88,70 +102,66 @@ __global__ void __launch_bounds__(kThreads) select_kernel(ckv_shape s, const flo
           }
         }
       }
-    }
-    if (run_cnt) atomicAdd(&whist[warp][run_bin], run_cnt);
-    __syncthreads();
-    // 256 threads add the per-warp histograms, then warp 0 (lane i owns digits 8 i .. 8 i + 7) finds the
-    // digit d with count(digit > d) < want <= count(digit >= d)
-    if (threadIdx.x < 256) {
-      int tot = 0;
+      if (run_cnt) atomicAdd(&whist[warp][run_bin], run_cnt);
+      __syncthreads();
+      // 256 threads add the per-warp histograms, then warp 0 (lane i owns digits 8 i .. 8 i + 7) finds the
+      // digit d with count(digit > d) < want <= count(digit >= d)
+      if (threadIdx.x < 256) {
+        int tot = 0;
 #pragma unroll 8
-      for (int w = 0; w < kWarps; ++w) tot += whist[w][threadIdx.x];
-      totals[threadIdx.x] = tot;
-    }
-    __syncthreads();
-    if (warp == 0) {
-      int cnt[8], mine = 0;
-#pragma unroll
-      for (int e = 0; e < 8; ++e) cnt[e] = totals[8 * lane + e], mine += cnt[e];
-      // above = number of matching keys in the digits of higher lanes
-      int incl = mine;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int x = __shfl_down_sync(0xffffffffu, incl, o);
-        if (lane + o < 32) incl += x;
+        for (int w = 0; w < kWarps; ++w) tot += whist[w][threadIdx.x];
+        totals[threadIdx.x] = tot;
       }
-      int above = incl - mine;
-      if (above < want && incl >= want) {   // the digit lies in this lane's range: exactly one lane
-        int dgt = 7;
-        for (; dgt > 0; --dgt) {
-          if (above + cnt[dgt] >= want) break;
-          above += cnt[dgt];
+      __syncthreads();
+      if (warp == 0) {
+        int cnt[8], mine = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) cnt[i] = totals[8 * lane + i], mine += cnt[i];
+        int incl = mine;   // matching keys in this lane's digits and in those of higher lanes
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int x = __shfl_down_sync(0xffffffffu, incl, o);
+          if (lane + o < 32) incl += x;
         }
-        sh_prefix = prefix | ((uint32_t)(8 * lane + dgt) << shift);
-        sh_want = want - above;
+        int above = incl - mine;
+        if (above < want && incl >= want) {   // the digit lies in this lane's range: exactly one lane
+          int dgt = 7;
+          for (; dgt > 0; --dgt) {
+            if (above + cnt[dgt] >= want) break;
+            above += cnt[dgt];
+          }
+          sh_prefix = prefix | ((uint32_t)(8 * lane + dgt) << shift);
+          sh_want = want - above;
+        }
       }
+      __syncthreads();
+      prefix = sh_prefix;
+      want = sh_want;
+      mask |= 0xffu << shift;
+      __syncthreads();
     }
-    __syncthreads();
-    prefix = sh_prefix;
-    want = sh_want;
-    mask |= 0xffu << shift;
-    __syncthreads();
   }
 
-  // ordered compaction
+  // ordered compaction.  First the per-warp totals of keys above and equal to the k-th ...
   int gt = 0, eq = 0;
   if (kCached) {
 #pragma unroll
-    for (int j = 0; j < kCache; ++j)
-      if (t0 + j < t1) gt += keys[j] > prefix, eq += keys[j] == prefix;
+    for (int j = 0; j < kCache; ++j) gt += keys[j] > prefix, eq += keys[j] == prefix;
   } else {
-    for (int t = t0; t < t1; ++t) {
+    for (int j = 0; j < chunk; ++j) {
+      const int t = base + 32 * j;
+      if (t >= wend) break;
       const uint32_t key = key_of(sc[t]);
-      gt += key > prefix;
-      eq += key == prefix;
+      gt += key > prefix, eq += key == prefix;
     }
   }
-  int gt_inc = gt, eq_inc = eq;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const int a = __shfl_up_sync(0xffffffffu, gt_inc, o), b = __shfl_up_sync(0xffffffffu, eq_inc, o);
-    if (lane >= o) gt_inc += a, eq_inc += b;
-  }
-  if (lane == 31) warp_gt[warp] = gt_inc, warp_eq[warp] = eq_inc;
+  gt = __reduce_add_sync(0xffffffffu, gt);
+  eq = __reduce_add_sync(0xffffffffu, eq);
   __syncthreads();
-  if (warp == 0) {
-    int a = warp_gt[lane], b = warp_eq[lane];
+  if (lane == 0) warp_gt[warp] = gt, warp_eq[warp] = eq;
+  __syncthreads();
+  if (warp == 0) {   // exclusive scan over the warps
+    const int a = warp_gt[lane], b = warp_eq[lane];
     int ai = a, bi = b;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -160,24 +170,35 @@ __global__ void __launch_bounds__(kThreads) select_kernel(ckv_shape s, const flo
     }
     warp_gt[lane] = ai - a;
     warp_eq[lane] = bi - b;
+    if (lane == 31) sh_want = e - ai;   // keys equal to the k-th that are kept: k minus all keys above it
   }
   __syncthreads();
-  int gt_before = warp_gt[warp] + gt_inc - gt, eq_before = warp_eq[warp] + eq_inc - eq;
-  auto place = [&](uint32_t key, int t) {
-    if (key > prefix) {
-      out[gt_before + min(eq_before, want)] = t;
-      ++gt_before;
-    } else if (key == prefix) {
-      if (eq_before < want) out[gt_before + eq_before] = t;
-      ++eq_before;
+  want = sh_want;
+  // ... then, row by row of the warp's range, ballots give every kept position its rank
+  int gt_run = warp_gt[warp], eq_run = warp_eq[warp];
+  const unsigned lt = (1u << lane) - 1u;
+  auto place_row = [&](uint32_t key, bool valid, int t) {
+    const unsigned gm = __ballot_sync(0xffffffffu, valid && key > prefix);
+    const unsigned em = __ballot_sync(0xffffffffu, valid && key == prefix);
+    const int gt_before = gt_run + __popc(gm & lt), eq_before = eq_run + __popc(em & lt);
+    if (valid) {
+      if (key > prefix) out[gt_before + min(eq_before, want)] = t;
+      else if (key == prefix && eq_before < want) out[gt_before + eq_before] = t;
     }
+    gt_run += __popc(gm), eq_run += __popc(em);
   };
   if (kCached) {
 #pragma unroll
-    for (int j = 0; j < kCache; ++j)
-      if (t0 + j < t1) place(keys[j], t0 + j);
+    for (int j = 0; j < kCache; ++j) {
+      const int t = base + 32 * j;
+      place_row(keys[j], j < chunk && t < wend, t);
+    }
   } else {
-    for (int t = t0; t < t1; ++t) place(key_of(sc[t]), t);
+    for (int j = 0; j < chunk; ++j) {
+      const int t = base + 32 * j;
+      const bool valid = t < wend;
+      place_row(valid ? key_of(sc[t]) : 0u, valid, t);
+    }
   }
 }
 
