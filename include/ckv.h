@@ -190,6 +190,12 @@ ckv_status ckv_device_status(const void* ws, void* stream);
  * returns the previous setting, or -1 for an invalid value. */
 int ckv_set_score_path(int path);
 
+/* Timing hook: when both are non-null cudaEvent_t handles (created with timing enabled, owned by the
+ * caller), every later ckv_score / ckv_compress call that runs the tensor-core scan records
+ * start_event just before and stop_event just after that kernel's launch, on the call's stream, so
+ * that the scan can be timed inside a fused call.  Pass nulls to switch it off.  Process-wide. */
+void ckv_set_scan_events(void* start_event, void* stop_event);
+
 /* Diagnostic knobs of the tensor-core scan's schedule (process-wide; results do not depend on them):
  *   "run_tiles"      key tiles per run, the unit CTAs take work in (1..64, default 8);
  *   "l2_hints"       1 (default): first-pass K loads ask L2 to keep their lines and second-pass loads

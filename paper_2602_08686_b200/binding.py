@@ -64,6 +64,8 @@ def lib() -> C.CDLL:
         L.ckv_compress.argtypes = [shp, prm, vp, vp, vp, fp, fp, vp, vp, i32p, i32p, i32p, fp, i32p, fp, vp, sz, vp]
         L.ckv_compress_host.argtypes = [shp, prm, vp, vp, vp, fp, fp, vp, vp, i32p, i32p, i32p, vp, sz, vp, sz, vp]
         L.ckv_device_status.argtypes = [vp, vp]
+        L.ckv_set_scan_events.argtypes = [vp, vp]
+        L.ckv_set_scan_events.restype = None
         L.ckv_set_tunable.argtypes = [C.c_char_p, C.c_int]
         L.ckv_set_tunable.restype = C.c_int
         L.ckv_kernel_launches.restype = C.c_int64
@@ -88,6 +90,14 @@ def ckv_version() -> int:
 def ckv_set_score_path(path: int) -> int:
     """0 automatic, 1 plain kernels, 2 tensor-core kernel required; returns the previous setting."""
     return int(lib().ckv_set_score_path(int(path)))
+
+
+def ckv_set_scan_events(start, stop) -> None:
+    """Timing hook: torch.cuda.Event objects (timing enabled, already recorded once so that their handles
+    exist) recorded around the tensor-core scan of every later call; ``None, None`` switches it off."""
+    h0 = None if start is None else C.c_void_p(start.cuda_event)
+    h1 = None if stop is None else C.c_void_p(stop.cuda_event)
+    lib().ckv_set_scan_events(h0, h1)
 
 
 def ckv_set_tunable(name: str, value: int) -> int:

@@ -9,6 +9,7 @@ namespace ckv {
 
 static std::atomic<int64_t> g_launches{0};
 static std::atomic<int> g_score_path{0};  // 0 = automatic, 1 = plain kernels, 2 = tensor-core kernel
+static std::atomic<cudaEvent_t> g_scan_start{nullptr}, g_scan_stop{nullptr};  // see ckv_set_scan_events
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
 static size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
@@ -112,9 +113,12 @@ static ckv_status score_impl(const ckv_shape& s, const ckv_params& p, const void
   const int path = g_score_path.load(std::memory_order_relaxed);
   const bool tc_ok = score_tc_supported(s) && s.seq_len >= 128;
   if (path == 2 && !tc_ok) return CKV_ERR_UNSUPPORTED;
+  const cudaEvent_t ev0 = g_scan_start.load(), ev1 = g_scan_stop.load();
   if (tc_ok && path != 1) {
+    if (ev0) CKV_CUDA(cudaEventRecord(ev0, st));
     CKV_CUDA(launch_score_tc(s, q, k, csum, ws + w.tc_part, ws + w.tc_stat, reinterpret_cast<int*>(ws + w.tc_flags),
                              reinterpret_cast<int*>(ws + w.status), st));
+    if (ev1) CKV_CUDA(cudaEventRecord(ev1, st));
   } else {
     CKV_CUDA(launch_score_plain(s, q, k, csum, reinterpret_cast<float2*>(ws + w.part),
                                 reinterpret_cast<float2*>(ws + w.stat), w.nblk, st));
@@ -296,6 +300,11 @@ ckv_status ckv_device_status(const void* ws, void* stream) {
 int ckv_set_score_path(int path) {
   if (path < 0 || path > 2) return -1;
   return g_score_path.exchange(path, std::memory_order_relaxed);
+}
+
+void ckv_set_scan_events(void* start_event, void* stop_event) {
+  g_scan_start.store((cudaEvent_t)start_event);
+  g_scan_stop.store((cudaEvent_t)stop_event);
 }
 
 int ckv_set_tunable(const char* name, int value) {
