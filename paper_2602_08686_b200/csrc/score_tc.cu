@@ -234,22 +234,31 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-// 2^x for x <= 0 on the FMA and integer pipes (the exponential unit is the scan's busiest pipe, so a
-// share of the exponentials goes here instead): x = n + f with n = round(x), f in [-0.5, 0.5];
-// 2^f by a degree-4 polynomial fitted for relative error (3e-6); 2^n by adding n to the exponent field.
-// Inputs below -125 are raised to -125 (2^-125 stands in for zero).
-__device__ __forceinline__ float ex2_poly(float x) {
-  x = fmaxf(x, -125.f);
-  const float t = x + 12582912.f;            // 1.5 * 2^23: the low mantissa bits of t hold n
-  const float f = x - (t - 12582912.f);
-  float p = fmaf(f, 9.582851277e-03f, 5.590642810e-02f);
-  p = fmaf(f, p, 2.402409867e-01f);
-  p = fmaf(f, p, 6.931241930e-01f);
-  p = fmaf(f, p, 1.f);
-  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+// Two-wide fp32 arithmetic (one instruction for a pair of values) and a three-input maximum: the
+// consumer loops are bound by instruction issue, and these halve the multiply-add, add and max counts.
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
 }
-// Which of the 32 values of a TMEM slice take the polynomial instead of the exponential unit.
-__device__ __forceinline__ constexpr bool use_poly(int jj) { return (jj & 3) == 3; }
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
 
 __device__ __forceinline__ int ld_acquire(const int* p) {
   int v;
@@ -673,15 +682,19 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           }
           float mx[4] = {v[0], v[1], v[2], v[3]};
 #pragma unroll
-          for (int jj = 4; jj < 32; ++jj) mx[jj & 3] = fmaxf(mx[jj & 3], v[jj]);
-          const float m_new = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * kScale, m_run);
-          const float negm = -m_new;
-          float sum[4] = {l_run * ex2(m_run - m_new), 0.f, 0.f, 0.f};
+          for (int pr = 2; pr < 16; ++pr) mx[pr & 3] = max3(mx[pr & 3], v[2 * pr], v[2 * pr + 1]);
+          const float m_new = fmaxf(max3(mx[0], mx[1], mx[2]) * kScale, fmaxf(mx[3] * kScale, m_run));
+          const uint64_t negm2 = pack2(-m_new, -m_new), scale2 = pack2(kScale, kScale);
+          uint64_t sum2[2] = {pack2(l_run * ex2(m_run - m_new), 0.f), pack2(0.f, 0.f)};
 #pragma unroll
-          for (int jj = 0; jj < 32; ++jj) {
-            const float x = fmaf(v[jj], kScale, negm);
-            sum[jj & 3] += use_poly(jj) ? ex2_poly(x) : ex2(x);
+          for (int jj = 0; jj < 32; jj += 2) {
+            float x0, x1;
+            unpack2(fma2(pack2(v[jj], v[jj + 1]), scale2, negm2), x0, x1);
+            sum2[(jj >> 1) & 1] = add2(sum2[(jj >> 1) & 1], pack2(ex2(x0), ex2(x1)));
           }
+          float sum[4];
+          unpack2(sum2[0], sum[0], sum[1]);
+          unpack2(sum2[1], sum[2], sum[3]);
           l_run = (sum[0] + sum[1]) + (sum[2] + sum[3]);
           m_run = m_new;
         }
@@ -714,25 +727,30 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         for (int cc = 0; cc < 4; ++cc) {
           float v[32];
           tmem_ld32(taddr + cc * 32, v);
-          float acc[kHeadsPerSlice][2];
+          uint64_t acc2[kHeadsPerSlice];   // per head of the slice: two running sums
 #pragma unroll
-          for (int hh = 0; hh < kHeadsPerSlice; ++hh) acc[hh][0] = acc[hh][1] = 0.f;
+          for (int hh = 0; hh < kHeadsPerSlice; ++hh) acc2[hh] = pack2(0.f, 0.f);
+          const uint64_t scale2 = pack2(kScale, kScale);
 #pragma unroll
           for (int j4 = 0; j4 < 8; ++j4) {
             const float4 b4 = reinterpret_cast<const float4*>(nb)[cc * 8 + j4];
-            const float bb[4] = {b4.x, b4.y, b4.z, b4.w};
+            const uint64_t bb2[2] = {pack2(b4.x, b4.y), pack2(b4.z, b4.w)};
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const int jj = j4 * 4 + e;
-              const float x = fmaf(v[jj], kScale, bb[e]);
-              float p = use_poly(jj) ? ex2_poly(x) : ex2(x);
+            for (int e2 = 0; e2 < 2; ++e2) {
+              const int jj = j4 * 4 + 2 * e2;
+              float x0, x1;
+              unpack2(fma2(pack2(v[jj], v[jj + 1]), scale2, bb2[e2]), x0, x1);
+              float p0 = ex2(x0), p1 = ex2(x1);
               if (tail) {
-                const int i = (cc * 32 + jj) % W;
-                if (t > a.n + i) p = 0.f;
+                if (t > a.n + (cc * 32 + jj) % W) p0 = 0.f;
+                if (t > a.n + (cc * 32 + jj + 1) % W) p1 = 0.f;
               }
-              acc[W >= 32 ? 0 : jj / W][e & 1] += p;
+              acc2[W >= 32 ? 0 : jj / W] = add2(acc2[W >= 32 ? 0 : jj / W], pack2(p0, p1));
             }
           }
+          float acc[kHeadsPerSlice][2];
+#pragma unroll
+          for (int hh = 0; hh < kHeadsPerSlice; ++hh) unpack2(acc2[hh], acc[hh][0], acc[hh][1]);
           if (cc == 3) {  // all bias reads and TMEM loads of this sub-item are done
             tc_fence_before();
             __syncwarp();
