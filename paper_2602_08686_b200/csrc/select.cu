@@ -6,8 +6,9 @@
 // positions w * 32 * chunk + 32 j + l, so that every load is coalesced and a ballot per j gives the
 // order inside the warp's range.  When a head's prefix fits (chunk <= 32) the keys stay in registers
 // and the search takes one bit per step: count the keys at or above the candidate (a compare per key,
-// one warp reduction, one barrier).  Longer prefixes use 8-bit digits with per-warp histograms and
-// re-read the scores in every pass.
+// one warp reduction, one barrier) until the keys that can still be the k-th fit one per thread; these
+// are then copied to shared memory and the remaining bits cost one ballot per warp and step.  Longer
+// prefixes use 8-bit digits with per-warp histograms and re-read the scores in every pass.
 #include "ckv_common.cuh"
 
 namespace ckv {
@@ -31,6 +32,8 @@ __global__ void __launch_bounds__(kThreads) select_kernel(ckv_shape s, const flo
   __shared__ int whist[kCached ? 1 : kWarps][256];   // 8-bit path: one histogram per warp
   __shared__ int totals[256];
   __shared__ int wcnt[2][kWarps];
+  __shared__ uint32_t list[kCached ? kThreads : 1];   // keys of the narrowed range
+  __shared__ int list_fill;
   __shared__ uint32_t sh_prefix;
   __shared__ int sh_want;
   __shared__ int warp_gt[kWarps], warp_eq[kWarps];
@@ -42,6 +45,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(ckv_shape s, const flo
   const float* sc = scores + ((int64_t)u * Hkv + g) * n;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
+  if (threadIdx.x == 0) list_fill = 0;
   for (int i = threadIdx.x; i < W; i += kThreads) out[e + i] = n + i;
   if (e <= 0) return;
   if (e >= n) {
@@ -64,21 +68,64 @@ __global__ void __launch_bounds__(kThreads) select_kernel(ckv_shape s, const flo
   uint32_t prefix = 0;
   int want = e;
   if (kCached) {
-    // one bit per step: the k-th largest key is the largest value v with #{keys >= v} >= k
-    for (int bit = 31; bit >= 0; --bit) {
+    // One bit per step: the k-th largest key is the largest value v with #{keys >= v} >= k.  The keys that
+    // can still be the k-th form the range [prefix, prefix + 2^(bit+1)); its size follows from the counts.
+    // While the range holds more keys than the CTA has threads, a step compares all cached keys; then the
+    // range is copied to shared memory, one key per thread, and the remaining steps cost a ballot each.
+    int above = 0;        // keys above the range: at or above every candidate inside it
+    int in_range = n;
+    int bit = 31, par = 0;
+    for (; bit >= 0 && in_range > kThreads; --bit, par ^= 1) {
       const uint32_t cand = prefix | (1u << bit);
       int c[4] = {0, 0, 0, 0};
 #pragma unroll
       for (int j = 0; j < kCache; ++j) c[j & 3] += keys[j] >= cand;
       const int cw = __reduce_add_sync(0xffffffffu, (c[0] + c[1]) + (c[2] + c[3]));
-      if (lane == 0) wcnt[0][warp] = cw;
-      __syncthreads();
-      if (warp == 0) {
-        const int tot = __reduce_add_sync(0xffffffffu, wcnt[0][lane]);
-        if (lane == 0) wcnt[1][0] = tot;
+      if (lane == 0) wcnt[par][warp] = cw;
+      __syncthreads();   // the other buffer is written in the next step, this one again only after that barrier
+      const int tot = __reduce_add_sync(0xffffffffu, wcnt[par][lane]);
+      if (tot >= e) {
+        prefix = cand;
+        in_range = tot - above;
+      } else {
+        in_range -= tot - above;
+        above = tot;
+      }
+    }
+    if (bit >= 0) {
+      const int sh = bit + 1;   // bits [31, sh) of the k-th key are known
+      __syncthreads();          // list_fill is zero for every warp
+      int m = 0;
+#pragma unroll
+      for (int j = 0; j < kCache; ++j) {
+        const bool valid = j < chunk && base + 32 * j < wend;
+        m += valid && (sh >= 32 || (keys[j] >> sh) == (prefix >> sh));
+      }
+      int incl = m;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int x = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += x;
+      }
+      int wbase = 0;
+      if (lane == 31 && incl) wbase = atomicAdd(&list_fill, incl);   // list order does not matter
+      int pos = __shfl_sync(0xffffffffu, wbase, 31) + incl - m;
+      if (m) {
+#pragma unroll
+        for (int j = 0; j < kCache; ++j) {
+          const bool valid = j < chunk && base + 32 * j < wend;
+          if (valid && (sh >= 32 || (keys[j] >> sh) == (prefix >> sh))) list[min(pos++, kThreads - 1)] = keys[j];
+        }
       }
       __syncthreads();
-      if (wcnt[1][0] >= e) prefix = cand;
+      const uint32_t ck = (int)threadIdx.x < min(list_fill, kThreads) ? list[threadIdx.x] : 0u;
+      for (; bit >= 0; --bit, par ^= 1) {
+        const uint32_t cand = prefix | (1u << bit);
+        const unsigned b = __ballot_sync(0xffffffffu, ck >= cand);
+        if (lane == 0) wcnt[par][warp] = __popc(b);
+        __syncthreads();
+        if (above + __reduce_add_sync(0xffffffffu, wcnt[par][lane]) >= e) prefix = cand;
+      }
     }
   } else {
     // 8 bits per pass from the top: after the loop `prefix` is the key of the e-th largest score

@@ -332,6 +332,41 @@ def test_select_exact_ties_and_extremes(B):
     assert idx[0, :8].tolist() == list(range(8))
 
 
+@pytest.mark.parametrize("n", [700, 1024, 1025, 5000, 32736, 32768, 40000])
+@pytest.mark.parametrize("dist", ["uniform", "lognormal", "tie_block", "signed"])
+def test_select_distributions(B, n, dist):
+    """ckv_select alone on score vectors whose candidate range narrows early, late or never."""
+    Nu, Hkv, W = 2, 4, 32
+    L = n + W
+    rng = np.random.default_rng(n * 7 + len(dist))
+    if dist == "uniform":
+        scores = rng.random((Nu, Hkv, n), dtype=np.float32)
+    elif dist == "lognormal":
+        scores = rng.lognormal(0.0, 3.0, (Nu, Hkv, n)).astype(np.float32)
+    elif dist == "signed":
+        scores = rng.standard_normal((Nu, Hkv, n)).astype(np.float32)
+    else:   # more equal scores at the cut than one key per thread can hold
+        scores = rng.random((Nu, Hkv, n), dtype=np.float32)
+        scores[:, :, rng.permutation(n)[: min(n - 8, 3000)]] = 0.75
+    a, b = min(n - 1, 480), max(1, n // 3)
+    b += (-(a + b + n)) % 4
+    budgets = np.array([[a, b, 1, n - 1], [n - 1, 1, b, a]], np.int32) + W
+    rows = int(budgets[0].sum())
+    assert rows % Hkv == 0 and int(budgets[1].sum()) == rows
+    offsets = np.concatenate([np.zeros((Nu, 1), np.int32), budgets.cumsum(1).astype(np.int32)], 1)
+    q = torch.zeros(Nu, Hkv, W, 128, dtype=torch.bfloat16, device="cuda")
+    k = torch.zeros(Nu, Hkv, L, 128, dtype=torch.bfloat16, device="cuda")
+    shape = B.make_shape(q, k)
+    params = B.make_params(B.Params(budget_per_head=rows // Hkv, floor_per_head=0), None, None)
+    ws = B.alloc_workspace(shape, params, "cuda")
+    idx = torch.full((Nu, rows), -1, dtype=torch.int32, device="cuda")
+    B.ckv_select(shape, params, torch.from_numpy(scores).cuda(), torch.from_numpy(budgets).cuda(),
+                 torch.from_numpy(offsets).cuda(), idx, ws)
+    prob = Problem(Nu, Hkv, Hkv, L, W, budget_per_head=rows // Hkv)
+    want = oracle.select(prob, scores.astype(np.float64), budgets, offsets)
+    np.testing.assert_array_equal(idx.cpu().numpy(), want)
+
+
 def test_strided_inputs(B):
     """K/V living inside a larger allocation (non-dense unit/head/token strides) give the same result."""
     cfg = gen.shrink(gen.CONFIGS["c2"], n_layers=2, n_q_heads=8, n_kv_heads=2, seq_len=700, budget_per_head=64,
