@@ -123,7 +123,7 @@ static ckv_status score_impl(const ckv_shape& s, const ckv_params& p, const void
     CKV_CUDA(launch_score_plain(s, q, k, csum, reinterpret_cast<float2*>(ws + w.part),
                                 reinterpret_cast<float2*>(ws + w.stat), w.nblk, st));
   }
-  CKV_CUDA(launch_epilogue(s, p, csum, head_w, scores, colmass, st));
+  CKV_CUDA(launch_epilogue(s, p, csum, head_w, scores, colmass, ws + w.ent_part, ws + w.bud_done, st));
   return CKV_OK;
 }
 
@@ -157,8 +157,9 @@ ckv_status ckv_budget(const ckv_shape* shape, const ckv_params* params, const fl
   CKV_TRY(check_ws(shape, params, ws, ws_bytes));
   const WsLayout w = ws_layout(*shape, *params);
   char* base = (char*)ws;
-  CKV_CUDA(launch_budget(*shape, *params, scores, colmass, sens, budgets, offsets, bucket, entropy,
-                         base + w.ent_part, base + w.cnt_part, base + w.bud_done, (cudaStream_t)stream));
+  CKV_CUDA(launch_entropy_partials(*shape, colmass, base + w.ent_part, base + w.bud_done, (cudaStream_t)stream));
+  CKV_CUDA(launch_budget(*shape, *params, scores, sens, budgets, offsets, bucket, entropy, base + w.ent_part,
+                         base + w.cnt_part, base + w.bud_done, (cudaStream_t)stream));
   return CKV_OK;
 }
 
@@ -201,8 +202,8 @@ ckv_status ckv_compress(const ckv_shape* shape, const ckv_params* params, const 
   int32_t* bucket = bucket_or_null ? bucket_or_null : reinterpret_cast<int32_t*>(base + w.bucket);
   float* entropy = entropy_or_null ? entropy_or_null : reinterpret_cast<float*>(base + w.entropy);
   CKV_TRY(score_impl(*shape, *params, q_win, k, head_w, scores, colmass, base, st));
-  CKV_CUDA(launch_budget(*shape, *params, scores, colmass, sens, budgets, offsets, bucket, entropy,
-                         base + w.ent_part, base + w.cnt_part, base + w.bud_done, st));
+  CKV_CUDA(launch_budget(*shape, *params, scores, sens, budgets, offsets, bucket, entropy, base + w.ent_part,
+                         base + w.cnt_part, base + w.bud_done, st));
   CKV_CUDA(launch_select(*shape, *params, scores, budgets, offsets, indices, st));
   CKV_CUDA(launch_gather(*shape, *params, k, v, indices, offsets, k_out, v_out, st));
   return CKV_OK;

@@ -11,6 +11,8 @@ constexpr int kHeadDim = 128;
 constexpr int kMaxWindow = 64;
 constexpr int kMaxKvHeads = 64;
 constexpr int kPlainKeysPerBlock = 256;  // keys per CTA in the plain (SIMT) score kernels
+constexpr int kEntSpan = 512;            // positions per entropy partial of the budget stage
+constexpr int kCountSpan = 8192;         // scores per counting CTA of the budget stage
 
 // log2(e): the softmax is evaluated in base 2, x = (q.k) * log2(e) / sqrt(d)
 constexpr float kLog2e = 1.4426950408889634f;
@@ -28,7 +30,7 @@ struct WsLayout {
   size_t tc_part;  // float2 [C, T+2, 128]     partial row statistics of the tensor-core scan
   size_t tc_stat;  // float2 [C, 128]          final row statistics per chunk
   size_t tc_flags; // int32 [C, 5]             completion counters and ready flags
-  size_t ent_part; // double [Nu, nblk]        entropy partials of the budget stage
+  size_t ent_part; // double [Nu, nblk]        entropy partials of the budget stage (nblk = ceil(L / kEntSpan))
   size_t cnt_part; // int32 [Nu, Hkv, S]       candidate counts per slice
   size_t bud_done; // int32 [Nu]               CTAs of the unit that have finished counting
   size_t total;
@@ -61,11 +63,16 @@ void count_launch(int n = 1);
 // Launchers; each returns cudaGetLastError() after queuing its kernels.
 cudaError_t launch_score_plain(const ckv_shape& s, const void* q, const void* k, float* csum, float2* part,
                                float2* stat, int nblk, cudaStream_t st);
+// The epilogue also leaves the budget stage's entropy partials (one per kEntSpan positions) and clears its
+// arrival counters; launch_entropy_partials does the same from a column mass the caller supplies.
 cudaError_t launch_epilogue(const ckv_shape& s, const ckv_params& p, const float* csum, const float* head_w,
-                            float* scores, float* colmass, cudaStream_t st);
-cudaError_t launch_budget(const ckv_shape& s, const ckv_params& p, const float* scores, const float* colmass,
-                          const float* sens, int32_t* budgets, int32_t* offsets, int32_t* bucket, float* entropy,
-                          void* ent_part, void* cnt_part, void* done, cudaStream_t st);
+                            float* scores, float* colmass, void* ent_part, void* done, cudaStream_t st);
+cudaError_t launch_entropy_partials(const ckv_shape& s, const float* colmass, void* ent_part, void* done,
+                                    cudaStream_t st);
+// Expects the entropy partials and cleared counters of one of the two launchers above.
+cudaError_t launch_budget(const ckv_shape& s, const ckv_params& p, const float* scores, const float* sens,
+                          int32_t* budgets, int32_t* offsets, int32_t* bucket, float* entropy, void* ent_part,
+                          void* cnt_part, void* done, cudaStream_t st);
 cudaError_t launch_select(const ckv_shape& s, const ckv_params& p, const float* scores, const int32_t* budgets,
                           const int32_t* offsets, int32_t* indices, cudaStream_t st);
 cudaError_t launch_gather(const ckv_shape& s, const ckv_params& p, const void* k, const void* v,

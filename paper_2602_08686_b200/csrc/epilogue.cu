@@ -1,5 +1,6 @@
-// Pooling, head-table weighting and group max (Eq. 4's L/W scale, Eq. 6 inside a GQA group), and
-// the unit's column mass for the entropy of Eq. 7, in one pass over the per-head column sums.
+// Pooling, head-table weighting and group max (Eq. 4's L/W scale, Eq. 6 inside a GQA group), the
+// unit's column mass and the per-CTA partial sums of its entropy (Eq. 7), in one pass over the
+// per-head column sums.
 #include "ckv_common.cuh"
 
 namespace ckv {
@@ -9,6 +10,43 @@ constexpr int kThreads = 128;
 constexpr int kPerThread = 4;                    // consecutive positions per thread
 constexpr int kSpan = kThreads * kPerThread;     // positions per CTA
 constexpr int kHeadBatch = 8;                    // heads staged in shared memory at a time
+static_assert(kSpan == kEntSpan, "one entropy partial per CTA");
+
+// Sum over the CTA's positions of -p ln p with p = mass / (W H); thread i holds positions 4 i .. 4 i + 3 and
+// passes zero for those past the end.  Fixed order: the thread's four terms, a shuffle tree, the warps in
+// index order.  Every thread must call; thread 0 gets the sum.
+__device__ __forceinline__ double entropy_partial(const float (&mass)[kPerThread], double norm) {
+  __shared__ double warp_sum[kThreads / 32];
+  double acc = 0.0;
+#pragma unroll
+  for (int e = 0; e < kPerThread; ++e) {
+    const double pt = (double)mass[e] * norm;
+    if (pt > 0.0) acc -= pt * log(pt);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if ((threadIdx.x & 31) == 0) warp_sum[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  double tot = 0.0;
+  if (threadIdx.x == 0)
+    for (int w = 0; w < kThreads / 32; ++w) tot += warp_sum[w];
+  return tot;
+}
+
+// The same partials from a column mass that is already in memory (the stand-alone budget call).
+__global__ void __launch_bounds__(kThreads) entropy_partials(ckv_shape s, const float* __restrict__ colmass,
+                                                             double* __restrict__ ent_part,
+                                                             int* __restrict__ done) {
+  const int u = blockIdx.y, L = s.seq_len, tb = blockIdx.x * kSpan + threadIdx.x * kPerThread;
+  float mass[kPerThread];
+#pragma unroll
+  for (int e = 0; e < kPerThread; ++e) mass[e] = tb + e < L ? colmass[(int64_t)u * L + tb + e] : 0.f;
+  const double tot = entropy_partial(mass, 1.0 / ((double)s.window * (double)s.n_q_heads));
+  if (threadIdx.x == 0) {
+    ent_part[(int64_t)u * gridDim.x + blockIdx.x] = tot;
+    if (blockIdx.x == 0) done[u] = 0;
+  }
+}
 
 // One CTA owns kSpan consecutive positions t of one unit and walks over all query heads:
 //   scores[u,g,t] = max_{h in g} head_w[h] * pool((L/W) c_h)[t]   for t < n  (pooling never looks past n)
@@ -20,7 +58,9 @@ __global__ void __launch_bounds__(kThreads) pool_weight_max_mass(ckv_shape s, ck
                                                                  const float* __restrict__ csum,
                                                                  const float* __restrict__ head_w,
                                                                  float* __restrict__ scores,
-                                                                 float* __restrict__ colmass) {
+                                                                 float* __restrict__ colmass,
+                                                                 double* __restrict__ ent_part,
+                                                                 int* __restrict__ done) {
   constexpr int kHalo = (R + 3) / 4 * 4;           // halo rounded up so that every thread's window is 16-byte aligned
   constexpr int kWidth = kSpan + 2 * kHalo;        // staged positions t0 - kHalo .. t0 + kSpan + kHalo - 1
   constexpr int kWin = kPerThread + 2 * kHalo;     // values a thread reads: c_h[tb - kHalo .. tb + 3 + kHalo]
@@ -102,33 +142,50 @@ __global__ void __launch_bounds__(kThreads) pool_weight_max_mass(ckv_shape s, ck
     }
   }
 #pragma unroll
-  for (int e = 0; e < kPerThread; ++e)
+  for (int e = 0; e < kPerThread; ++e) {
     if (tb + e < L) colmass[(int64_t)u * L + tb + e] = mass[e];
+    else mass[e] = 0.f;
+  }
+  const double tot = entropy_partial(mass, 1.0 / ((double)s.window * (double)H));
+  if (threadIdx.x == 0) {
+    ent_part[(int64_t)u * gridDim.x + blockIdx.x] = tot;
+    if (blockIdx.x == 0) done[u] = 0;
+  }
 }
 
 template <int R>
 void launch_r(bool avg, dim3 grid, cudaStream_t st, const ckv_shape& s, const ckv_params& p, const float* csum,
-              const float* head_w, float* scores, float* colmass) {
-  if (avg) pool_weight_max_mass<R, true><<<grid, kThreads, 0, st>>>(s, p, csum, head_w, scores, colmass);
-  else pool_weight_max_mass<R, false><<<grid, kThreads, 0, st>>>(s, p, csum, head_w, scores, colmass);
+              const float* head_w, float* scores, float* colmass, double* ent, int* done) {
+  if (avg) pool_weight_max_mass<R, true><<<grid, kThreads, 0, st>>>(s, p, csum, head_w, scores, colmass, ent, done);
+  else pool_weight_max_mass<R, false><<<grid, kThreads, 0, st>>>(s, p, csum, head_w, scores, colmass, ent, done);
 }
 
 }  // namespace
 
+cudaError_t launch_entropy_partials(const ckv_shape& s, const float* colmass, void* ent_part, void* done,
+                                    cudaStream_t st) {
+  dim3 grid((s.seq_len + kSpan - 1) / kSpan, s.n_units);
+  entropy_partials<<<grid, kThreads, 0, st>>>(s, colmass, (double*)ent_part, (int*)done);
+  count_launch();
+  return cudaGetLastError();
+}
+
 cudaError_t launch_epilogue(const ckv_shape& s, const ckv_params& p, const float* csum, const float* head_w,
-                            float* scores, float* colmass, cudaStream_t st) {
+                            float* scores, float* colmass, void* ent_part, void* done, cudaStream_t st) {
+  double* ent = (double*)ent_part;
+  int* dn = (int*)done;
   dim3 grid((s.seq_len + kSpan - 1) / kSpan, s.n_units);
   const int r = (p.pool_kind == CKV_POOL_NONE) ? 0 : p.pool_size / 2;
   const bool avg = p.pool_kind == CKV_POOL_AVG && r > 0;
   switch (r) {
-    case 0: launch_r<0>(false, grid, st, s, p, csum, head_w, scores, colmass); break;
-    case 1: launch_r<1>(avg, grid, st, s, p, csum, head_w, scores, colmass); break;
-    case 2: launch_r<2>(avg, grid, st, s, p, csum, head_w, scores, colmass); break;
-    case 3: launch_r<3>(avg, grid, st, s, p, csum, head_w, scores, colmass); break;
-    case 4: launch_r<4>(avg, grid, st, s, p, csum, head_w, scores, colmass); break;
-    case 5: launch_r<5>(avg, grid, st, s, p, csum, head_w, scores, colmass); break;
-    case 6: launch_r<6>(avg, grid, st, s, p, csum, head_w, scores, colmass); break;
-    default: launch_r<7>(avg, grid, st, s, p, csum, head_w, scores, colmass); break;
+    case 0: launch_r<0>(false, grid, st, s, p, csum, head_w, scores, colmass, ent, dn); break;
+    case 1: launch_r<1>(avg, grid, st, s, p, csum, head_w, scores, colmass, ent, dn); break;
+    case 2: launch_r<2>(avg, grid, st, s, p, csum, head_w, scores, colmass, ent, dn); break;
+    case 3: launch_r<3>(avg, grid, st, s, p, csum, head_w, scores, colmass, ent, dn); break;
+    case 4: launch_r<4>(avg, grid, st, s, p, csum, head_w, scores, colmass, ent, dn); break;
+    case 5: launch_r<5>(avg, grid, st, s, p, csum, head_w, scores, colmass, ent, dn); break;
+    case 6: launch_r<6>(avg, grid, st, s, p, csum, head_w, scores, colmass, ent, dn); break;
+    default: launch_r<7>(avg, grid, st, s, p, csum, head_w, scores, colmass, ent, dn); break;
   }
   count_launch();
   return cudaGetLastError();
