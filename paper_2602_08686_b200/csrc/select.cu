@@ -3,16 +3,21 @@
 // equal scores are resolved toward the lowest index, and the observation window is appended.
 // One CTA per (unit, KV head); integer work only, bit-exact and deterministic.
 //
-// Prefixes of up to 32768 positions take the bit-sliced kernel: thread i owns the 32 consecutive
-// positions from 32 i.  The scores are read coalesced, turned into ordered keys and staged in shared
-// memory, from where every thread fetches its own 128-byte line; a 32 x 32 bit transpose in registers
-// leaves plane b holding bit b of the thread's 32 keys.  A search step then costs a few logic
+// The bit-sliced kernel: thread i of a CTA owns the 32 consecutive positions from 32 i, a CTA 32768
+// positions, and prefixes of up to eight times that are spread over the CTAs of a thread-block
+// cluster.  The scores are read coalesced, turned into ordered keys and staged in shared memory, from
+// where every thread fetches its own 128-byte line; a 32 x 32 bit transpose in registers leaves plane
+// b holding bit b of the thread's 32 keys.  A search step then costs a few logic
 // operations and population counts per thread whatever the number of keys, so two bits are decided per
 // CTA-wide reduction (16 reductions for the whole key).  The search ends with one mask of the keys above
 // the k-th and one of the keys equal to it; their population counts, scanned over the threads in position
 // order, place every kept position.
 //
-// Longer prefixes use 8-bit digits with per-warp histograms and re-read the scores in every pass.
+// Still longer prefixes use 8-bit digits with per-warp histograms and re-read the scores in every pass.
+#include <cooperative_groups.h>
+
+#include <algorithm>
+
 #include "ckv_common.cuh"
 
 namespace ckv {
@@ -48,37 +53,51 @@ __device__ __forceinline__ void transpose32(uint32_t (&a)[32]) {
   }
 }
 
+// kCluster CTAs of one thread-block cluster share a head: CTA r holds the positions from r * kSlicedMax.
+// Every warp then sends its counts to all CTAs of the cluster through distributed shared memory and the
+// step's barrier spans the cluster.
+template <int kCluster>
 __global__ void __launch_bounds__(kThreads) select_sliced_kernel(ckv_shape s, const float* __restrict__ scores,
                                                                  const int32_t* __restrict__ budgets,
                                                                  const int32_t* __restrict__ offsets,
                                                                  int32_t* __restrict__ indices) {
   extern __shared__ __align__(16) uint32_t stage[];   // [warps in use][1024] keys in position order
-  __shared__ uint2 wcnt[2][kWarps];
+  __shared__ uint2 wcnt[2][kCluster][kWarps];
   __shared__ uint32_t wtot[kWarps];
+  __shared__ uint32_t ctot[kCluster];
   const int Hkv = s.n_kv_heads, W = s.window, n = s.seq_len - W;
-  const int u = blockIdx.x / Hkv, g = blockIdx.x % Hkv;
+  const int head = blockIdx.x / kCluster, rank = blockIdx.x % kCluster;
+  const int u = head / Hkv, g = head % Hkv;
   const int e = budgets[(int64_t)u * Hkv + g] - W;
   const int64_t rows_per_unit = offsets[(int64_t)u * (Hkv + 1) + Hkv];
   int32_t* out = indices + (int64_t)u * rows_per_unit + offsets[(int64_t)u * (Hkv + 1) + g];
   const float* sc = scores + ((int64_t)u * Hkv + g) * n;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int cbase = rank * kSlicedMax;                      // first position of this CTA
+  const int first = cbase + 32 * (int)threadIdx.x;          // first position of this thread
 
-  for (int i = threadIdx.x; i < W; i += kThreads) out[e + i] = n + i;
+  // the branches below are taken by all CTAs of a cluster alike
+  if (rank == 0)
+    for (int i = threadIdx.x; i < W; i += kThreads) out[e + i] = n + i;
   if (e <= 0) return;
   if (e >= n) {
-    for (int t = threadIdx.x; t < n; t += kThreads) out[t] = t;
+    for (int t = cbase + threadIdx.x; t < min(n, cbase + kSlicedMax); t += kThreads) out[t] = t;
     return;
   }
+  auto step_barrier = [&]() {
+    if constexpr (kCluster == 1) __syncthreads();
+    else cooperative_groups::this_cluster().sync();
+  };
 
-  // a[31 - k] = key of position 32 * tid + (k + 4 * lane) % 32: the 16-byte pieces of the thread's line are
+  // a[31 - k] = key of position first + (k + 4 * lane) % 32: the 16-byte pieces of the thread's line are
   // fetched in an order rotated by the lane so that a quarter warp touches every bank once
   uint32_t a[32];
   const int wbase = warp * 1024;
-  if (wbase < n) {
+  if (cbase + wbase < n) {
     uint32_t* ws = stage + wbase;
 #pragma unroll
     for (int j = 0; j < 32; ++j) {
-      const int t = wbase + 32 * j + lane;
+      const int t = cbase + wbase + 32 * j + lane;
       ws[32 * j + lane] = t < n ? key_of(sc[t]) : 0u;
     }
     __syncwarp();
@@ -94,13 +113,13 @@ __global__ void __launch_bounds__(kThreads) select_sliced_kernel(ckv_shape s, co
   }
   transpose32(a);   // a[31 - b] bit k = bit b of the k-th fetched key
 
-  // positions of the thread that exist, in fetch order (bit k <-> position 32 tid + (k + 4 lane) % 32)
+  // positions of the thread that exist, in fetch order (bit k <-> position first + (k + 4 lane) % 32)
   const int rot = (4 * lane) & 31;
-  const int have = min(max(n - 32 * (int)threadIdx.x, 0), 32);
+  const int have = min(max(n - first, 0), 32);
   const uint32_t valid_pos = have >= 32 ? 0xffffffffu : ((1u << have) - 1u);
   uint32_t alive = __funnelshift_r(valid_pos, valid_pos, rot);   // keys equal to the decided bits so far
   uint32_t gt = 0u;                                              // keys above the k-th
-  int above = 0;                                                 // their number in the whole CTA
+  int above = 0;                                                 // their number over the whole head
 #pragma unroll
   for (int st = 0; st < 16; ++st) {
     const uint32_t p1 = a[2 * st], p0 = a[2 * st + 1];   // planes of bits 31 - 2 st and 30 - 2 st
@@ -108,12 +127,28 @@ __global__ void __launch_bounds__(kThreads) select_sliced_kernel(ckv_shape s, co
     const uint32_t h1 = h & p0, l1 = l & p0;
     const uint32_t r1 = __reduce_add_sync(0xffffffffu, (uint32_t)__popc(h1) | ((uint32_t)__popc(h) << 16));
     const uint32_t r2 = __reduce_add_sync(0xffffffffu, (uint32_t)__popc(l1));
-    if (lane == 0) wcnt[st & 1][warp] = make_uint2(r1, r2);
-    __syncthreads();   // the other buffer is written in the next step, this one again only after that barrier
-    const uint2 w = wcnt[st & 1][lane];
-    const uint32_t t1 = __reduce_add_sync(0xffffffffu, w.x);
-    const int t01 = (int)__reduce_add_sync(0xffffffffu, w.y);
-    const int t11 = (int)(t1 & 0xffffu), t1x = (int)(t1 >> 16);
+    // the other buffer is written in the next step, this one again only after that step's barrier
+    if constexpr (kCluster == 1) {
+      if (lane == 0) wcnt[st & 1][0][warp] = make_uint2(r1, r2);
+    } else {
+      if (lane < kCluster)
+        *cooperative_groups::this_cluster().map_shared_rank(&wcnt[st & 1][rank][warp], lane) = make_uint2(r1, r2);
+    }
+    step_barrier();
+    uint32_t wx = 0, wy = 0;   // lane l adds warp l of every CTA: both 16-bit fields stay below 2^14
+#pragma unroll
+    for (int c = 0; c < kCluster; ++c) {
+      const uint2 w = wcnt[st & 1][c][lane];
+      wx += w.x, wy += w.y;
+    }
+    int t11, t1x;
+    if constexpr (kCluster == 1) {
+      const uint32_t t1 = __reduce_add_sync(0xffffffffu, wx);
+      t11 = (int)(t1 & 0xffffu), t1x = (int)(t1 >> 16);
+    } else {
+      t11 = (int)__reduce_add_sync(0xffffffffu, wx & 0xffffu), t1x = (int)__reduce_add_sync(0xffffffffu, wx >> 16);
+    }
+    const int t01 = (int)__reduce_add_sync(0xffffffffu, wy);
     if (above + t11 >= e) {               // digit 11
       alive = h1;
     } else if (above + t1x >= e) {        // digit 10
@@ -136,17 +171,23 @@ __global__ void __launch_bounds__(kThreads) select_sliced_kernel(ckv_shape s, co
   }
   if (lane == 31) wtot[warp] = incl;
   __syncthreads();
-  const uint32_t before = __reduce_add_sync(0xffffffffu, lane < warp ? wtot[lane] : 0u) + incl - mine;
-  const int gt_before = (int)(before & 0xffffu), eq_before = (int)(before >> 16);
+  const uint32_t wt = wtot[lane];
+  const uint32_t before = __reduce_add_sync(0xffffffffu, lane < warp ? wt : 0u) + incl - mine;
+  int gt_before = (int)(before & 0xffffu), eq_before = (int)(before >> 16);
+  if constexpr (kCluster > 1) {   // kept keys of the CTAs holding lower positions
+    const uint32_t total = __reduce_add_sync(0xffffffffu, wt);
+    if (warp == 0 && lane < kCluster) *cooperative_groups::this_cluster().map_shared_rank(&ctot[rank], lane) = total;
+    cooperative_groups::this_cluster().sync();
+    for (int c = 0; c < rank; ++c) gt_before += (int)(ctot[c] & 0xffffu), eq_before += (int)(ctot[c] >> 16);
+  }
   uint32_t m = gtp | eqp;
   while (m) {
     const int j = __ffs((int)m) - 1;
     const uint32_t bit = 1u << j;
     m &= m - 1u;
     const int gb = gt_before + __popc(gtp & (bit - 1u)), eb = eq_before + __popc(eqp & (bit - 1u));
-    const int t = 32 * (int)threadIdx.x + j;
-    if (gtp & bit) out[gb + min(eb, want)] = t;
-    else if (eb < want) out[gb + eb] = t;
+    if (gtp & bit) out[gb + min(eb, want)] = first + j;
+    else if (eb < want) out[gb + eb] = first + j;
   }
 }
 
@@ -287,23 +328,43 @@ __global__ void __launch_bounds__(kThreads) select_digit_kernel(ckv_shape s, con
   }
 }
 
+
+template <int kCluster>
+cudaError_t launch_sliced(const ckv_shape& s, int n, const float* scores, const int32_t* budgets,
+                          const int32_t* offsets, int32_t* indices, cudaStream_t st) {
+  const int per_cta = (n + kCluster - 1) / kCluster;   // staging covers the fullest CTA
+  const size_t smem = (size_t)((std::min(per_cta, kSlicedMax) + 1023) / 1024) * 1024 * sizeof(uint32_t);
+  cudaError_t e = cudaFuncSetAttribute(select_sliced_kernel<kCluster>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       kSlicedMax * (int)sizeof(uint32_t));
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)(s.n_units * s.n_kv_heads * kCluster));
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kCluster == 1 ? smem : kSlicedMax * sizeof(uint32_t);
+  cfg.stream = st;
+  cudaLaunchAttribute attr{};
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = kCluster, attr.val.clusterDim.y = 1, attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr, cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, select_sliced_kernel<kCluster>, s, scores, budgets, offsets, indices);
+}
+
 }  // namespace
 
 cudaError_t launch_select(const ckv_shape& s, const ckv_params&, const float* scores, const int32_t* budgets,
                           const int32_t* offsets, int32_t* indices, cudaStream_t st) {
   const int n = s.seq_len - s.window;
-  const int grid = s.n_units * s.n_kv_heads;
-  if (n <= kSlicedMax) {
-    const size_t smem = (size_t)((n + 1023) / 1024) * 1024 * sizeof(uint32_t);
-    cudaError_t e = cudaFuncSetAttribute(select_sliced_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         kSlicedMax * (int)sizeof(uint32_t));
-    if (e != cudaSuccess) return e;
-    select_sliced_kernel<<<grid, kThreads, smem, st>>>(s, scores, budgets, offsets, indices);
-  } else {
-    select_digit_kernel<<<grid, kThreads, 0, st>>>(s, scores, budgets, offsets, indices);
+  cudaError_t e;
+  if (n <= kSlicedMax) e = launch_sliced<1>(s, n, scores, budgets, offsets, indices, st);
+  else if (n <= 2 * kSlicedMax) e = launch_sliced<2>(s, n, scores, budgets, offsets, indices, st);
+  else if (n <= 4 * kSlicedMax) e = launch_sliced<4>(s, n, scores, budgets, offsets, indices, st);
+  else if (n <= 8 * kSlicedMax) e = launch_sliced<8>(s, n, scores, budgets, offsets, indices, st);
+  else {
+    select_digit_kernel<<<s.n_units * s.n_kv_heads, kThreads, 0, st>>>(s, scores, budgets, offsets, indices);
+    e = cudaGetLastError();
   }
   count_launch();
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace ckv

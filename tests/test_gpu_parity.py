@@ -332,10 +332,11 @@ def test_select_exact_ties_and_extremes(B):
     assert idx[0, :8].tolist() == list(range(8))
 
 
-@pytest.mark.parametrize("n", [700, 1024, 1025, 5000, 32736, 32768, 40000])
+@pytest.mark.parametrize("n", [700, 1024, 1025, 5000, 32736, 32768, 32769, 40000, 65536, 131040, 200000, 262145])
 @pytest.mark.parametrize("dist", ["uniform", "lognormal", "tie_block", "signed"])
 def test_select_distributions(B, n, dist):
-    """ckv_select alone on score vectors whose candidate range narrows early, late or never."""
+    """ckv_select alone: one CTA, clusters of 2, 4 and 8 CTAs and the digit path, on score vectors with few or
+    many equal values at the cut."""
     Nu, Hkv, W = 2, 4, 32
     L = n + W
     rng = np.random.default_rng(n * 7 + len(dist))
