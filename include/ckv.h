@@ -196,10 +196,16 @@ int ckv_set_score_path(int path);
  * that the scan can be timed inside a fused call.  Pass nulls to switch it off.  Process-wide. */
 void ckv_set_scan_events(void* start_event, void* stop_event);
 
-/* Diagnostic knobs of the tensor-core scan's schedule (process-wide; results do not depend on them):
+/* Diagnostic knobs of the tensor-core scan (process-wide; the scores do not depend on them):
  *   "run_tiles"      key tiles per run, the unit CTAs take work in (1..64, default 8);
  *   "l2_hints"       1 (default): first-pass K loads ask L2 to keep their lines and second-pass loads
- *                    release them; 0: no hints.
+ *                    release them; 0: no hints;
+ *   "group_fuse"     1 (default): where a KV group's query heads fill one 128-row block and the pooling
+ *                    is max or none, the scan itself takes the weighted maximum over the group's heads
+ *                    (Eq. 6) and adds their column mass, and the pooling runs on that one row per group;
+ *                    the scores are bit-identical to the per-head order of operations for head_w >= 0,
+ *                    the column mass may differ in the last bit (heads are added group by group);
+ *                    0: always write per-head column sums.
  * Returns the previous value, or -1 for an unknown name or a value out of range. */
 int ckv_set_tunable(const char* name, int value);
 

@@ -1,5 +1,6 @@
 // Host side of the C ABI: argument validation, work-space layout and the launch sequences.
 #include <atomic>
+#include <string>
 #include <cstring>
 #include <mutex>
 
@@ -9,6 +10,7 @@ namespace ckv {
 
 static std::atomic<int64_t> g_launches{0};
 static std::atomic<int> g_score_path{0};  // 0 = automatic, 1 = plain kernels, 2 = tensor-core kernel
+static std::atomic<int> g_group_fuse{1};  // 1: the scan writes per-group maxima and masses where it can
 static std::atomic<cudaEvent_t> g_scan_start{nullptr}, g_scan_stop{nullptr};  // see ckv_set_scan_events
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
@@ -115,10 +117,18 @@ static ckv_status score_impl(const ckv_shape& s, const ckv_params& p, const void
   if (path == 2 && !tc_ok) return CKV_ERR_UNSUPPORTED;
   const cudaEvent_t ev0 = g_scan_start.load(), ev1 = g_scan_stop.load();
   if (tc_ok && path != 1) {
+    // grouped output where it applies: both arrays fit the per-head region (at least two heads per group)
+    TcGrouped grp{csum, csum + (int64_t)s.n_units * s.n_kv_heads * s.seq_len, head_w, p.head_w_stride_unit};
+    const bool grouped = score_tc_groupable(s, p) && g_group_fuse.load(std::memory_order_relaxed) != 0;
     if (ev0) CKV_CUDA(cudaEventRecord(ev0, st));
-    CKV_CUDA(launch_score_tc(s, q, k, csum, ws + w.tc_part, ws + w.tc_stat, reinterpret_cast<int*>(ws + w.tc_flags),
-                             reinterpret_cast<int*>(ws + w.status), st));
+    CKV_CUDA(launch_score_tc(s, q, k, csum, grouped ? &grp : nullptr, ws + w.tc_part, ws + w.tc_stat,
+                             reinterpret_cast<int*>(ws + w.tc_flags), reinterpret_cast<int*>(ws + w.status), st));
     if (ev1) CKV_CUDA(cudaEventRecord(ev1, st));
+    if (grouped) {
+      CKV_CUDA(launch_epilogue_grouped(s, p, grp.zgrp, grp.mgrp, scores, colmass, ws + w.ent_part, ws + w.bud_done,
+                                       st));
+      return CKV_OK;
+    }
   } else {
     CKV_CUDA(launch_score_plain(s, q, k, csum, reinterpret_cast<float2*>(ws + w.part),
                                 reinterpret_cast<float2*>(ws + w.stat), w.nblk, st));
@@ -310,6 +320,7 @@ void ckv_set_scan_events(void* start_event, void* stop_event) {
 
 int ckv_set_tunable(const char* name, int value) {
   if (!name) return -1;
+  if (std::string(name) == "group_fuse") return g_group_fuse.exchange(value != 0 ? 1 : 0);
   return set_tc_tunable(name, value);
 }
 

@@ -53,8 +53,19 @@ struct TcLayout {
 TcLayout tc_layout(const ckv_shape& s);
 bool score_tc_supported(const ckv_shape& s);
 int set_tc_tunable(const char* name, int value);
-cudaError_t launch_score_tc(const ckv_shape& s, const void* q, const void* k, float* csum, void* part, void* stat,
-                            int* flags, int* status, cudaStream_t st);
+// Grouped output of the scan (see score_tc.cu): per KV group the weighted maximum over its query heads and
+// their summed column mass, [Nu, Hkv, L] each, instead of the per-head column sums.  Possible when a group's
+// heads fill one row block, there are at least two of them and the pooling is max or none; requires
+// head weights >= 0 (a maximum commutes with the pooling only then).
+struct TcGrouped {
+  float* zgrp;
+  float* mgrp;
+  const float* head_w;
+  int64_t hw_stride;
+};
+bool score_tc_groupable(const ckv_shape& s, const ckv_params& p);
+cudaError_t launch_score_tc(const ckv_shape& s, const void* q, const void* k, float* csum, const TcGrouped* grp,
+                            void* part, void* stat, int* flags, int* status, cudaStream_t st);
 
 WsLayout ws_layout(const ckv_shape& s, const ckv_params& p);
 
@@ -67,6 +78,9 @@ cudaError_t launch_score_plain(const ckv_shape& s, const void* q, const void* k,
 // arrival counters; launch_entropy_partials does the same from a column mass the caller supplies.
 cudaError_t launch_epilogue(const ckv_shape& s, const ckv_params& p, const float* csum, const float* head_w,
                             float* scores, float* colmass, void* ent_part, void* done, cudaStream_t st);
+// The same from the scan's grouped output: pooling of zgrp inside the prefix, column mass from mgrp.
+cudaError_t launch_epilogue_grouped(const ckv_shape& s, const ckv_params& p, const float* zgrp, const float* mgrp,
+                                    float* scores, float* colmass, void* ent_part, void* done, cudaStream_t st);
 cudaError_t launch_entropy_partials(const ckv_shape& s, const float* colmass, void* ent_part, void* done,
                                     cudaStream_t st);
 // Expects the entropy partials and cleared counters of one of the two launchers above.

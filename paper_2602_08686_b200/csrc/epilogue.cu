@@ -53,9 +53,13 @@ __global__ void __launch_bounds__(kThreads) entropy_partials(ckv_shape s, const 
 //   colmass[u,t]  = sum_h c_h[t]                                    for t < L  (heads added in index order)
 // R is the pooling radius (window 2R + 1); AVG counts positions outside the prefix as zeros and divides
 // by the window size, MAX ignores them.
-template <int R, bool AVG>
+// GROUPED: csum holds one row per KV group that is already weighted, scaled and maximised over the
+// group's heads (max pooling commutes with that for weights >= 0), and gmass the groups' column mass:
+//   scores[u,g,t] = pool(csum[u,g])[t],   colmass[u,t] = sum_g gmass[u,g,t]   (groups in index order)
+template <int R, bool AVG, bool GROUPED>
 __global__ void __launch_bounds__(kThreads) pool_weight_max_mass(ckv_shape s, ckv_params p,
                                                                  const float* __restrict__ csum,
+                                                                 const float* __restrict__ gmass,
                                                                  const float* __restrict__ head_w,
                                                                  float* __restrict__ scores,
                                                                  float* __restrict__ colmass,
@@ -65,9 +69,10 @@ __global__ void __launch_bounds__(kThreads) pool_weight_max_mass(ckv_shape s, ck
   constexpr int kWidth = kSpan + 2 * kHalo;        // staged positions t0 - kHalo .. t0 + kSpan + kHalo - 1
   constexpr int kWin = kPerThread + 2 * kHalo;     // values a thread reads: c_h[tb - kHalo .. tb + 3 + kHalo]
   __shared__ __align__(16) float tile[kHeadBatch][kWidth];
-  const int L = s.seq_len, n = L - s.window, H = s.n_q_heads, G = H / s.n_kv_heads;
+  const int L = s.seq_len, n = L - s.window;
+  const int H = GROUPED ? s.n_kv_heads : s.n_q_heads, G = GROUPED ? 1 : H / s.n_kv_heads;   // rows of csum
   const int u = blockIdx.y, t0 = blockIdx.x * kSpan, tb = t0 + threadIdx.x * kPerThread;
-  const float scale = (float)L / (float)s.window;
+  const float scale = GROUPED ? 1.f : (float)L / (float)s.window;
   const float inv_size = 1.f / (float)(2 * R + 1);
   const float pad = AVG ? 0.f : -INFINITY;
   const float* hw = head_w + (int64_t)u * p.head_w_stride_unit;
@@ -83,6 +88,15 @@ __global__ void __launch_bounds__(kThreads) pool_weight_max_mass(ckv_shape s, ck
       // all loads of the batch first, then the stores: the loads are independent and overlap
       constexpr int kIters = (kWidth + kThreads - 1) / kThreads;
       float buf[kHeadBatch][kIters];
+      float gm[GROUPED ? kHeadBatch : 1][kPerThread];
+      if (GROUPED) {
+#pragma unroll
+        for (int hh = 0; hh < kHeadBatch; ++hh) {
+          const float* m = gmass + ((int64_t)u * H + h0 + (hh < nh ? hh : 0)) * L;
+#pragma unroll
+          for (int e = 0; e < kPerThread; ++e) gm[hh][e] = (hh < nh && (interior || tb + e < L)) ? m[tb + e] : 0.f;
+        }
+      }
 #pragma unroll
       for (int hh = 0; hh < kHeadBatch; ++hh) {
         const float* c = csum + ((int64_t)u * H + h0 + (hh < nh ? hh : 0)) * L;
@@ -101,6 +115,12 @@ __global__ void __launch_bounds__(kThreads) pool_weight_max_mass(ckv_shape s, ck
           if (i < kWidth) tile[hh][i] = buf[hh][it];
         }
       }
+      if (GROUPED) {
+#pragma unroll
+        for (int hh = 0; hh < kHeadBatch; ++hh)
+#pragma unroll
+          for (int e = 0; e < kPerThread; ++e) mass[e] += gm[hh][e];   // zero beyond the batch
+      }
     }
     __syncthreads();
     for (int hh = 0; hh < nh; ++hh) {
@@ -112,9 +132,11 @@ __global__ void __launch_bounds__(kThreads) pool_weight_max_mass(ckv_shape s, ck
         const float4 x = src[q4];
         win[4 * q4] = x.x, win[4 * q4 + 1] = x.y, win[4 * q4 + 2] = x.z, win[4 * q4 + 3] = x.w;
       }
+      if (!GROUPED) {
 #pragma unroll
-      for (int e = 0; e < kPerThread; ++e)
-        if (interior || tb + e < L) mass[e] += win[kHalo + e];
+        for (int e = 0; e < kPerThread; ++e)
+          if (interior || tb + e < L) mass[e] += win[kHalo + e];
+      }
       if (!interior) {   // the pooling only sees the prefix [0, n)
 #pragma unroll
         for (int i = 0; i < kWin; ++i) {
@@ -122,7 +144,7 @@ __global__ void __launch_bounds__(kThreads) pool_weight_max_mass(ckv_shape s, ck
           if (tt < 0 || tt >= n) win[i] = pad;
         }
       }
-      const float w = hw[h];
+      const float w = GROUPED ? 1.f : hw[h];
 #pragma unroll
       for (int e = 0; e < kPerThread; ++e) {
         float v = win[kHalo + e - R];
@@ -146,7 +168,7 @@ __global__ void __launch_bounds__(kThreads) pool_weight_max_mass(ckv_shape s, ck
     if (tb + e < L) colmass[(int64_t)u * L + tb + e] = mass[e];
     else mass[e] = 0.f;
   }
-  const double tot = entropy_partial(mass, 1.0 / ((double)s.window * (double)H));
+  const double tot = entropy_partial(mass, 1.0 / ((double)s.window * (double)s.n_q_heads));
   if (threadIdx.x == 0) {
     ent_part[(int64_t)u * gridDim.x + blockIdx.x] = tot;
     if (blockIdx.x == 0) done[u] = 0;
@@ -156,8 +178,16 @@ __global__ void __launch_bounds__(kThreads) pool_weight_max_mass(ckv_shape s, ck
 template <int R>
 void launch_r(bool avg, dim3 grid, cudaStream_t st, const ckv_shape& s, const ckv_params& p, const float* csum,
               const float* head_w, float* scores, float* colmass, double* ent, int* done) {
-  if (avg) pool_weight_max_mass<R, true><<<grid, kThreads, 0, st>>>(s, p, csum, head_w, scores, colmass, ent, done);
-  else pool_weight_max_mass<R, false><<<grid, kThreads, 0, st>>>(s, p, csum, head_w, scores, colmass, ent, done);
+  if (avg)
+    pool_weight_max_mass<R, true, false><<<grid, kThreads, 0, st>>>(s, p, csum, nullptr, head_w, scores, colmass, ent, done);
+  else
+    pool_weight_max_mass<R, false, false><<<grid, kThreads, 0, st>>>(s, p, csum, nullptr, head_w, scores, colmass, ent, done);
+}
+
+template <int R>
+void launch_g(dim3 grid, cudaStream_t st, const ckv_shape& s, const ckv_params& p, const float* zgrp,
+              const float* mgrp, float* scores, float* colmass, double* ent, int* done) {
+  pool_weight_max_mass<R, false, true><<<grid, kThreads, 0, st>>>(s, p, zgrp, mgrp, nullptr, scores, colmass, ent, done);
 }
 
 }  // namespace
@@ -186,6 +216,26 @@ cudaError_t launch_epilogue(const ckv_shape& s, const ckv_params& p, const float
     case 5: launch_r<5>(avg, grid, st, s, p, csum, head_w, scores, colmass, ent, dn); break;
     case 6: launch_r<6>(avg, grid, st, s, p, csum, head_w, scores, colmass, ent, dn); break;
     default: launch_r<7>(avg, grid, st, s, p, csum, head_w, scores, colmass, ent, dn); break;
+  }
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_epilogue_grouped(const ckv_shape& s, const ckv_params& p, const float* zgrp, const float* mgrp,
+                                    float* scores, float* colmass, void* ent_part, void* done, cudaStream_t st) {
+  double* ent = (double*)ent_part;
+  int* dn = (int*)done;
+  dim3 grid((s.seq_len + kSpan - 1) / kSpan, s.n_units);
+  const int r = (p.pool_kind == CKV_POOL_NONE) ? 0 : p.pool_size / 2;
+  switch (r) {
+    case 0: launch_g<0>(grid, st, s, p, zgrp, mgrp, scores, colmass, ent, dn); break;
+    case 1: launch_g<1>(grid, st, s, p, zgrp, mgrp, scores, colmass, ent, dn); break;
+    case 2: launch_g<2>(grid, st, s, p, zgrp, mgrp, scores, colmass, ent, dn); break;
+    case 3: launch_g<3>(grid, st, s, p, zgrp, mgrp, scores, colmass, ent, dn); break;
+    case 4: launch_g<4>(grid, st, s, p, zgrp, mgrp, scores, colmass, ent, dn); break;
+    case 5: launch_g<5>(grid, st, s, p, zgrp, mgrp, scores, colmass, ent, dn); break;
+    case 6: launch_g<6>(grid, st, s, p, zgrp, mgrp, scores, colmass, ent, dn); break;
+    default: launch_g<7>(grid, st, s, p, zgrp, mgrp, scores, colmass, ent, dn); break;
   }
   count_launch();
   return cudaGetLastError();

@@ -74,6 +74,14 @@ struct TcArgs {
   uint32_t q_bytes;     // bytes of one Q block load
   int q_split;          // the Q box holds fewer than 128 rows: its two halves are loaded separately
   float* csum;
+  // Grouped output (a KV group's query heads fill one row block, max or no pooling): instead of the
+  // per-head column sums c_h[t], P2 writes zgrp[u, g, t] = max_h head_w[h] * ((L / W) c_h[t]) and
+  // mgrp[u, g, t] = sum_h c_h[t] (heads in index order); both are [Nu, Hkv, L].  Null zgrp: per-head output.
+  float* zgrp;
+  float* mgrp;
+  const float* head_w;
+  int64_t hw_stride;    // elements between the head tables of consecutive units (0: one shared table)
+  float lw_scale;       // L / W
   float2* part;         // [C][ppr*RPC][128] partial (row max, row sum) per run and consumer group
   float2* stat;         // [C][128]          (row max, row max + log2 row sum)
   int* done;            // [C][4]
@@ -101,7 +109,9 @@ struct __align__(16) Desc {
   int chunk;
   int tile;       // key tile within the chunk
   int part_slot;  // P1: where this group's pair of the run goes, or -1 while the run goes on
+                  // P2: offset of the row block's first head in the head-weight table
   int first;      // P1: this group's first tile of the run (reset the running pair)
+                  // P2: index (u * Hkv + g) of the KV group
   int head0;      // P2: index (u * H + head) of the first query head of the row block
   int n_heads;    // P2: query heads of the row block that exist
   int nbias_buf;  // P2: which bias vector belongs to the tile's chunk
@@ -461,9 +471,14 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         const int tile = ln.ric * a.run + ln.k;
         // the n-th load of a lane's rows (n = 0, 1, ...) completes phase n of its barrier: wait for parity n & 1
         const int q_phase = (ln.q_loads - 1) & 1;
-        d[0] = make_int4(ln.type | (q_phase << 9), ln.chunk, tile,
-                         (ln.k + 2 >= ln.tr) ? ln.ric * a.ppr + (ln.k & 1) : -1);
-        d[1] = make_int4(ln.k < 2, ln.u * a.H + ln.head0, ln.heads, ln.gen % kBiasBufs);
+        if (ln.type == kP1) {
+          d[0] = make_int4(ln.type | (q_phase << 9), ln.chunk, tile,
+                           (ln.k + 2 >= ln.tr) ? ln.ric * a.ppr + (ln.k & 1) : -1);
+          d[1] = make_int4(ln.k < 2, 0, 0, 0);
+        } else {
+          d[0] = make_int4(ln.type | (q_phase << 9), ln.chunk, tile, ln.u * (int)a.hw_stride + ln.head0);
+          d[1] = make_int4(ln.u * a.Hkv + ln.g, ln.u * a.H + ln.head0, ln.heads, ln.gen % kBiasBufs);
+        }
         mbar_arrive_expect_tx(bar, kTileBytes);
         if (reload) {
           const uint32_t qbar = smem_u32(&sm.q_full[lane_id]);
@@ -722,7 +737,25 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         const float* nb = sm.nbias[d.nbias_buf];
         constexpr int kHeadsPerSlice = W >= 32 ? 1 : 32 / W;  // heads inside one 32-row TMEM load
         float* out = a.csum + (int64_t)d.head0 * a.L + t;
-        float head_acc = 0.f;
+        const bool grouped = a.zgrp != nullptr;
+        const float* hw = a.head_w + d.part_slot;
+        float wv[4] = {0.f, 0.f, 0.f, 0.f};   // the block's head weights when it holds at most four heads
+        if (grouped && W >= 32) {
+#pragma unroll
+          for (int hl = 0; hl < 128 / (W >= 32 ? W : 32); ++hl)
+            if (hl < d.n_heads) wv[hl] = __ldg(hw + hl);
+        }
+        float head_acc = 0.f, zmax = -INFINITY, msum = 0.f;
+        // a finished head: its column sum goes to memory, or into the group's weighted maximum and mass
+        auto head_done = [&](int hl, float c, float w) {
+          if (hl >= d.n_heads) return;
+          if (!grouped) {
+            if (t < a.L) out[(int64_t)hl * a.L] = c;
+          } else {
+            zmax = fmaxf(zmax, w * (c * a.lw_scale));
+            msum += c;
+          }
+        };
 #pragma unroll 1
         for (int cc = 0; cc < 4; ++cc) {
           float v[32];
@@ -761,16 +794,21 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
             const int rows_done = (cc + 1) * 32;
             if (rows_done % W == 0) {
               const int hl = rows_done / W - 1;
-              if (hl < d.n_heads && t < a.L) out[(int64_t)hl * a.L] = head_acc;
+              head_done(hl, head_acc, hl == 0 ? wv[0] : hl == 1 ? wv[1] : hl == 2 ? wv[2] : wv[3]);
               head_acc = 0.f;
             }
           } else {
 #pragma unroll
             for (int hh = 0; hh < kHeadsPerSlice; ++hh) {
               const int hl = cc * kHeadsPerSlice + hh;
-              if (hl < d.n_heads && t < a.L) out[(int64_t)hl * a.L] = acc[hh][0] + acc[hh][1];
+              head_done(hl, acc[hh][0] + acc[hh][1], grouped && hl < d.n_heads ? __ldg(hw + hl) : 0.f);
             }
           }
+        }
+        if (grouped && t < a.L) {
+          const int64_t o = (int64_t)d.first * a.L + t;
+          a.zgrp[o] = zmax;
+          a.mgrp[o] = msum;
         }
       }
       if (quad == 0 && lane == 0) TC_TRACE(5, j);
@@ -876,10 +914,19 @@ int set_tc_tunable(const char* name, int value) {
   return -1;
 }
 
-cudaError_t launch_score_tc(const ckv_shape& s, const void* q, const void* k, float* csum, void* part, void* stat,
-                            int* flags, int* status, cudaStream_t st) {
+bool score_tc_groupable(const ckv_shape& s, const ckv_params& p) {
+  const bool avg = p.pool_kind == CKV_POOL_AVG && p.pool_size / 2 > 0;
+  return score_tc_supported(s) && tc_layout(s).RB == 1 && s.n_q_heads >= 2 * s.n_kv_heads && !avg;
+}
+
+cudaError_t launch_score_tc(const ckv_shape& s, const void* q, const void* k, float* csum, const TcGrouped* grp,
+                            void* part, void* stat, int* flags, int* status, cudaStream_t st) {
   const TcLayout t = tc_layout(s);
   TcArgs a{};
+  if (grp) {
+    a.zgrp = grp->zgrp, a.mgrp = grp->mgrp, a.head_w = grp->head_w, a.hw_stride = grp->hw_stride;
+    a.lw_scale = (float)s.seq_len / (float)s.window;
+  }
   a.Nu = s.n_units, a.H = s.n_q_heads, a.Hkv = s.n_kv_heads, a.G = a.H / a.Hkv, a.L = s.seq_len, a.W = s.window;
   a.n = a.L - a.W;
   a.RB = t.RB, a.hpb = kTile / a.W, a.T = t.T, a.C = (int)t.C;

@@ -238,6 +238,31 @@ def test_tensor_core_path_is_taken_and_agrees_with_plain(B):
     assert rel < 1e-4, rel
 
 
+@pytest.mark.parametrize("G,W,pool_kind,pool_size", [(4, 32, 1, 7), (2, 64, 1, 3), (8, 16, 1, 5), (3, 16, 0, 1),
+                                                     (4, 16, 1, 15)])
+def test_grouped_scan_output_matches_per_head_output(B, G, W, pool_kind, pool_size):
+    """The scan's per-group maximum and mass (group_fuse) against its per-head column sums: the same scores
+    bit for bit (head_w >= 0), the same budgets and indices."""
+    cfg = gen.shrink(gen.CONFIGS["c2"], n_layers=2, n_q_heads=2 * G, n_kv_heads=2, seq_len=3000, window=W,
+                     pool_kind=pool_kind, pool_size=pool_size, budget_per_head=128, n_needles=8)
+    b = gen.make_batch(cfg, "cuda")
+    P = params_of(B, problem_of(cfg, 2))
+    prev_path = B.ckv_set_score_path(2)
+    prev = B.ckv_set_tunable("group_fuse", 1)
+    try:
+        fused = B.compress(b["q"], b["k"], b["v"], b["head_w"], b["sens"], P, want_scores=True)
+        assert B.ckv_device_status(fused["ws"]) == B.OK
+        B.ckv_set_tunable("group_fuse", 0)
+        plain = B.compress(b["q"], b["k"], b["v"], b["head_w"], b["sens"], P, want_scores=True)
+        assert B.ckv_device_status(plain["ws"]) == B.OK
+    finally:
+        B.ckv_set_tunable("group_fuse", prev)
+        B.ckv_set_score_path(prev_path)
+    assert torch.equal(fused["scores"], plain["scores"])
+    for key in ("budgets", "offsets", "indices"):
+        assert torch.equal(fused[key], plain[key]), key
+
+
 @pytest.mark.parametrize("G,W", [(1, 32), (2, 64), (3, 16), (9, 16), (5, 32)])
 def test_group_sizes_and_windows(B, G, W):
     """Row blocks: G*W below, equal to and above 128 rows (several blocks, the last one partial)."""
