@@ -695,28 +695,53 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_empty);
           }
-          float mx[4] = {v[0], v[1], v[2], v[3]};
+          // The running sum is kept relative to a reference m_run that need not be the row maximum: any
+          // reference gives the same (m, l) up to rounding as long as the sum stays inside the fp32 range.
+          // So the maximum is only taken on the run's first slice, or when a sum leaves that range.
+          const uint64_t scale2 = pack2(kScale, kScale);
+          auto slice_sum = [&](float ref) {
+            const uint64_t negm2 = pack2(-ref, -ref);
+            uint64_t sum2[2] = {pack2(0.f, 0.f), pack2(0.f, 0.f)};
 #pragma unroll
-          for (int pr = 2; pr < 16; ++pr) mx[pr & 3] = max3(mx[pr & 3], v[2 * pr], v[2 * pr + 1]);
-          const float m_new = fmaxf(max3(mx[0], mx[1], mx[2]) * kScale, fmaxf(mx[3] * kScale, m_run));
-          const uint64_t negm2 = pack2(-m_new, -m_new), scale2 = pack2(kScale, kScale);
-          uint64_t sum2[2] = {pack2(l_run * ex2(m_run - m_new), 0.f), pack2(0.f, 0.f)};
-#pragma unroll
-          for (int jj = 0; jj < 32; jj += 2) {
-            float x0, x1;
-            unpack2(fma2(pack2(v[jj], v[jj + 1]), scale2, negm2), x0, x1);
-            sum2[(jj >> 1) & 1] = add2(sum2[(jj >> 1) & 1], pack2(ex2(x0), ex2(x1)));
+            for (int jj = 0; jj < 32; jj += 2) {
+              float x0, x1;
+              unpack2(fma2(pack2(v[jj], v[jj + 1]), scale2, negm2), x0, x1);
+              sum2[(jj >> 1) & 1] = add2(sum2[(jj >> 1) & 1], pack2(ex2(x0), ex2(x1)));
+            }
+            float sum[4];
+            unpack2(sum2[0], sum[0], sum[1]);
+            unpack2(sum2[1], sum[2], sum[3]);
+            return (sum[0] + sum[1]) + (sum[2] + sum[3]);
+          };
+          float part = 0.f;
+          bool in_range = false;
+          if (!(d.first && cc == 0)) {
+            part = slice_sum(m_run);
+            in_range = l_run + part < 3.0e38f;   // false for infinities and NaNs too
           }
-          float sum[4];
-          unpack2(sum2[0], sum[0], sum[1]);
-          unpack2(sum2[1], sum[2], sum[3]);
-          l_run = (sum[0] + sum[1]) + (sum[2] + sum[3]);
-          m_run = m_new;
+          if (!in_range) {
+            float mx[4] = {v[0], v[1], v[2], v[3]};
+#pragma unroll
+            for (int pr = 2; pr < 16; ++pr) mx[pr & 3] = max3(mx[pr & 3], v[2 * pr], v[2 * pr + 1]);
+            const float m_new = fmaxf(max3(mx[0], mx[1], mx[2]) * kScale, fmaxf(mx[3] * kScale, m_run));
+            l_run *= ex2(m_run - m_new);
+            m_run = m_new;
+            part = slice_sum(m_run);
+          }
+          l_run += part;
         }
         if (d.part_slot >= 0) {
           // this group's last tile of the run: publish the pair; the last warp of the chunk's
           // quadrant merges all of them in slot order
-          a.part[((int64_t)d.chunk * (a.ppr * a.RPC) + d.part_slot) * kTile + row] = make_float2(m_run, l_run);
+          // (the pair is normalised to a sum in [1, 2), its power of two moved into the reference, so that the
+          // merge adds numbers of like size whatever the reference was)
+          float m_pub = m_run, l_pub = l_run;
+          if (l_run > 0.f) {
+            const int bits = __float_as_int(l_run);
+            m_pub = m_run + (float)((bits >> 23) - 127);
+            l_pub = __int_as_float((bits & 0x007fffff) | 0x3f800000);
+          }
+          a.part[((int64_t)d.chunk * (a.ppr * a.RPC) + d.part_slot) * kTile + row] = make_float2(m_pub, l_pub);
           __threadfence();
           __syncwarp();
           int prev = 0;

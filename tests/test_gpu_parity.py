@@ -238,6 +238,43 @@ def test_tensor_core_path_is_taken_and_agrees_with_plain(B):
     assert rel < 1e-4, rel
 
 
+@pytest.mark.parametrize("jump", [60.0, 140.0, 400.0])
+def test_logits_far_above_the_running_reference(B, jump):
+    """Keys whose logits exceed everything before them by `jump` powers of two: the scan's running sums are
+    kept relative to an early reference and must re-base when they leave the fp32 range (jump > 127)."""
+    Nu, H, Hkv, L, W = 2, 8, 2, 3000, 32
+    g = torch.Generator().manual_seed(int(jump))
+    u_dir = torch.zeros(128)
+    u_dir[:4] = 0.5                                  # unit vector
+    q = 0.3 * torch.randn(Nu, H, W, 128, generator=g) + 8.0 * u_dir
+    k = 0.3 * torch.randn(Nu, Hkv, L, 128, generator=g)
+    k -= (k @ u_dir)[..., None] * u_dir              # ordinary keys: no component along the queries' direction
+    amp = jump * math.sqrt(128.0) / (8.0 * math.log2(math.e))   # logit of a planted key ~ jump (base 2)
+    for t, f in ((700, 0.5), (1500, 1.0), (2600, 1.0), (2601, 0.98)):
+        k[:, :, t] += f * amp * u_dir
+    v = torch.randn(Nu, Hkv, L, 128, generator=g)
+    cfg = gen.shrink(gen.CONFIGS["c2"], n_layers=Nu, n_q_heads=H, n_kv_heads=Hkv, seq_len=L, window=W,
+                     budget_per_head=128, n_needles=0)
+    b = dict(q=q.bfloat16(), k=k.bfloat16(), v=v.bfloat16(), head_w=0.5 + torch.rand(Nu, H, generator=g),
+             sens=gen.make_sens(cfg))
+    prob = problem_of(cfg, Nu)
+    ref = oracle.score(prob, *(gen.as_numpy(b[x]) for x in ("q", "k", "head_w")))
+    for path in (2, 1):
+        prev = B.ckv_set_score_path(path)
+        try:
+            out = B.compress(b["q"].cuda(), b["k"].cuda(), b["v"].cuda(), b["head_w"].cuda(), b["sens"].cuda(),
+                             params_of(B, prob), want_scores=True)
+            assert B.ckv_device_status(out["ws"]) == B.OK
+        finally:
+            B.ckv_set_score_path(prev)
+        s = out["scores"].double().cpu().numpy()
+        assert np.isfinite(s).all()
+        big = ref[0] > 1e-30                          # below that both sides are zero to fp32
+        rel = np.abs(s - ref[0])[big] / ref[0][big]
+        assert rel.max() <= SCORE_RTOL, (path, rel.max())
+        assert np.abs(s[~big]).max(initial=0.0) <= 1e-30
+
+
 @pytest.mark.parametrize("G,W,pool_kind,pool_size", [(4, 32, 1, 7), (2, 64, 1, 3), (8, 16, 1, 5), (3, 16, 0, 1),
                                                      (4, 16, 1, 15)])
 def test_grouped_scan_output_matches_per_head_output(B, G, W, pool_kind, pool_size):
