@@ -238,6 +238,44 @@ def test_tensor_core_path_is_taken_and_agrees_with_plain(B):
     assert rel < 1e-4, rel
 
 
+@pytest.mark.parametrize("n_buckets,dup", [(1, False), (5, True), (16, False), (32, True), (40, False)])
+def test_fused_budget_equals_staged_budget(B, n_buckets, dup):
+    """The fused call's budget stage (entropy partials left by the pooling kernel) against ckv_budget on the
+    same scores and column mass (partials from its own kernel): same buckets, budgets and offsets for tables
+    of several sizes, with repeated thresholds and with scores equal to a threshold."""
+    cfg = gen.shrink(gen.CONFIGS["c2"], n_layers=3, n_q_heads=8, n_kv_heads=4, seq_len=2500, budget_per_head=96,
+                     n_needles=8, n_buckets=n_buckets)
+    b = gen.make_batch(cfg, "cuda")
+    sens = b["sens"].clone()
+    prob = problem_of(cfg, 3)
+    P = params_of(B, prob)
+    first = B.compress(b["q"], b["k"], b["v"], b["head_w"], sens, P, want_scores=True)
+    # thresholds taken from the scores themselves: candidates exist, and some scores equal the threshold
+    flat = first["scores"].flatten().sort(descending=True).values
+    picks = flat[torch.linspace(20, 2000, n_buckets).long()]
+    sens = picks[torch.randperm(n_buckets, generator=torch.Generator().manual_seed(3))].contiguous()
+    if dup and n_buckets > 2:
+        sens[1] = sens[0]
+        sens[-1] = sens[2]
+    for override in (-1, 0, n_buckets - 1):
+        prob_o = problem_of(cfg, 3, bucket_override=override)
+        P = params_of(B, prob_o)
+        out = B.compress(b["q"], b["k"], b["v"], b["head_w"], sens, P, want_scores=True)
+        shape = B.make_shape(b["q"], b["k"])
+        params = B.make_params(P, b["head_w"], sens)
+        ws = B.alloc_workspace(shape, params, "cuda")
+        scores = torch.empty_like(out["scores"])
+        colmass = torch.empty(3, cfg.seq_len, device="cuda")
+        B.ckv_score(shape, params, b["q"], b["k"], b["head_w"], scores, colmass, ws)
+        assert torch.equal(scores, out["scores"])
+        budgets, offsets = torch.zeros_like(out["budgets"]), torch.zeros_like(out["offsets"])
+        bucket, entropy = torch.zeros_like(out["bucket"]), torch.zeros_like(out["entropy"])
+        B.ckv_budget(shape, params, scores, colmass, sens, budgets, offsets, bucket, entropy, ws)
+        for key, val in (("bucket", bucket), ("budgets", budgets), ("offsets", offsets), ("entropy", entropy)):
+            assert torch.equal(out[key], val), (override, key, out[key], val)
+        assert len(set(out["budgets"].flatten().tolist())) > 1   # the thresholds do bite
+
+
 @pytest.mark.parametrize("jump", [60.0, 140.0, 400.0])
 def test_logits_far_above_the_running_reference(B, jump):
     """Keys whose logits exceed everything before them by `jump` powers of two: the scan's running sums are
