@@ -31,9 +31,10 @@ from paper_2602_08686_b200.sharding import max_over_ranks  # noqa: E402
 METRIC = "prefill_tokens_compressed_per_sec_per_layer"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one score_tc_kernel launch (ncu, see profiles/), keyed by
-# (workload, units); None where no capture of the current kernel exists
-SCAN_DRAM_TRAFFIC = {}
+# dram__bytes_read.sum + dram__bytes_write.sum of score_tc_kernel per unit, from an ncu capture of an 8-unit
+# launch of the workload's shape (profiles/score_tc_kernel_c2_8units.md); a launch's traffic is this times its
+# units (every unit streams its own K once per pass).  Workloads without a capture of the current kernel: none.
+SCAN_DRAM_TRAFFIC_PER_UNIT = {"c2": (1.011664e9 + 15.674112e6) / 8}
 
 
 def measured_peaks():
@@ -264,7 +265,8 @@ def main():
     peak, peak_kind = measured_peaks()
     k2_bytes, gather_bytes = algorithmic_bytes(cfg, n_units)
     scan_gbs = k2_bytes / (scan_ms * 1e-3) / 1e9
-    traffic = SCAN_DRAM_TRAFFIC.get((cfg.name, n_units))
+    traffic = SCAN_DRAM_TRAFFIC_PER_UNIT.get(cfg.name)
+    traffic = traffic * n_units if traffic is not None else None
     roofline = {"bound": "hbm", "kernel": "score_tc_kernel (window-score scan, both passes over K)",
                 "achieved": scan_gbs, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
                 "frac": scan_gbs / peak, "traffic": traffic,
