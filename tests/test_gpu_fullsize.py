@@ -1,0 +1,116 @@
+"""GPU parity at the full sizes of the five workloads, in the launch configuration bench.py times (one fused
+call over all units resident on the device).  The oracle is too slow for every unit, so it checks sampled units
+completely (scores, column mass, budgets, indices) and every unit is held to the properties that need no
+oracle: budgets sum to the total, windows kept, indices ascending, needles kept, gathered rows equal to the rows
+the indices name."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2602_08686_b200 import inputs as gen
+from test_gpu_parity import (SCORE_RTOL, check_bucket, check_selection_against_oracle, check_structure, params_of,
+                             problem_of)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2602_08686_b200 import binding
+    binding.lib()
+    assert torch.cuda.is_available()
+    return binding
+
+
+def needle_census(cfg, b, idx, bud, off):
+    """(planted, kept, lost) over the heads whose prefix budget covers all needle neighbourhoods and the sink's
+    (pooling spreads a needle's score over pool_size positions)."""
+    r, W = cfg.pool_size // 2, cfg.window
+    planted = kept = 0
+    lost = []
+    for u in range(idx.shape[0]):
+        for g in range(cfg.n_kv_heads):
+            needles = b["needles"][u, g].tolist()
+            hood = set(range(0, r + 1))
+            for t in needles:
+                hood |= set(range(t - r, t + r + 1))
+            if bud[u, g] - W >= len(hood):
+                s = set(idx[u, off[u, g]:off[u, g + 1]].tolist())
+                planted += len(needles)
+                kept += sum(int(t) in s for t in needles)
+                lost += [(u, g, int(t)) for t in needles if int(t) not in s]
+    return planted, kept, lost
+
+
+def run_full(B, cfg, units, sample):
+    """One fused call over `units`; oracle comparison on the positions `sample` of that list."""
+    b = gen.make_batch(cfg, "cuda", units)
+    Nu = len(units)
+    prob = problem_of(cfg, Nu)
+    out = B.compress(b["q"], b["k"], b["v"], b["head_w"], b["sens"], params_of(B, prob), want_scores=True)
+    assert B.ckv_device_status(out["ws"]) == B.OK
+    idx, bud, off = (out[x].cpu().numpy() for x in ("indices", "budgets", "offsets"))
+    check_structure(idx, bud, off, prob)
+    Hkv = cfg.n_kv_heads
+    # gather, every unit, on the device: row r of head g is K[u, g, idx[r]]
+    for u in range(Nu):
+        for g in range(Hkv):
+            sl = slice(int(off[u, g]), int(off[u, g + 1]))
+            rows = out["indices"][u, sl].long()
+            assert torch.equal(out["k_out"][u, sl], b["k"][u, g, rows])
+            assert torch.equal(out["v_out"][u, sl], b["v"][u, g, rows])
+    # sampled units against the oracle
+    for j in sample:
+        one = {x: b[x][j:j + 1].cpu() for x in ("q", "k", "head_w")}
+        prob1 = problem_of(cfg, 1)
+        sc, cm = oracle.score(prob1, *(gen.as_numpy(one[x]) for x in ("q", "k", "head_w")))
+        gs = out["scores"][j:j + 1].double().cpu().numpy()
+        rel = np.abs(gs - sc) / np.maximum(np.abs(sc), 1e-20)
+        assert rel.max() <= SCORE_RTOL, (j, rel.max())
+        ref = oracle.budget(prob1, sc, cm, gen.as_numpy(b["sens"]))
+        assert abs(float(out["entropy"][j]) - ref["entropy"][0]) <= 1e-4
+        check_bucket(out["bucket"][j:j + 1], ref, prob1)
+        # the oracle's budget step and selection on the GPU's own scores and bucket: exact
+        prob_b = problem_of(cfg, 1, bucket_override=int(out["bucket"][j]))
+        mine = oracle.budget(prob_b, gs, cm, gen.as_numpy(b["sens"]))
+        assert (mine["budgets"][0] == bud[j]).all()
+        np.testing.assert_array_equal(idx[j:j + 1], oracle.select(prob1, gs, bud[j:j + 1], off[j:j + 1]))
+        # and against the oracle's own scores: differences only inside the near-tie band
+        ref["scores"], ref["idx"] = sc, oracle.select(prob1, sc, ref["budgets"], ref["offsets"])
+        check_selection_against_oracle(idx[j:j + 1], bud[j:j + 1], off[j:j + 1], ref, prob1)
+    # planted needles, every unit.  A needle is aligned with one window query only, and where several needles of
+    # a head share that row its attention is split, so a few fall short of the cut at this scale (the oracle pins
+    # the strict form on small cases).  Under heavy-tailed key scales or average pooling other keys pass the
+    # needles by design of the workload; there the oracle comparison above is the check.
+    if not cfg.heavy_tail and cfg.pool_kind == 1:
+        planted, kept, lost = needle_census(cfg, b, idx, bud, off)
+        assert kept >= 0.99 * planted, (kept, planted, lost[:8])
+    del b, out
+    torch.cuda.empty_cache()
+
+
+def test_config2_full(B):
+    """32 layers of the Llama-3-8B shape at L 32768 in one call (the bench's step); units 0, 13 and 31 checked."""
+    cfg = gen.CONFIGS["c2"]
+    run_full(B, cfg, list(range(cfg.n_units)), [0, 13, 31])
+
+
+def test_config3_serving_batch(B):
+    """Batch 16: units of all sixteen sequences in one call (four layers each: 64 of the 512 units, 17 GB)."""
+    cfg = gen.CONFIGS["c3"]
+    units = [seq * cfg.n_layers + layer for seq in range(cfg.batch) for layer in (0, 9, 20, 31)]
+    run_full(B, cfg, units, [5, 62])
+
+
+def test_config4_full(B):
+    """L 131072, budget 2048, heavy-tailed keys: all 32 layers in one call; one unit checked against the oracle."""
+    cfg = gen.CONFIGS["c4"]
+    run_full(B, cfg, list(range(cfg.n_units)), [17])
+
+
+@pytest.mark.parametrize("L,budget", [(4096, 128), (16384, 512), (65536, 2048), (65536, 128)])
+def test_config5_sweep(B, L, budget):
+    """Qwen2.5-7B shape (GQA 7, W 64, avg pool 5, floor 8, low-reliability heads), batch 4 x 28 layers in one call."""
+    cfg = gen.shrink(gen.CONFIGS["c5"], seq_len=L, budget_per_head=budget)
+    run_full(B, cfg, list(range(cfg.n_units)), [3, 100] if L <= 16384 else [57])
