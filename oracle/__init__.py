@@ -39,7 +39,7 @@ class _Shape(C.Structure):
 class _Params(C.Structure):
     _fields_ = [(n, C.c_int32) for n in
                 ("pool_kind", "pool_size", "budget_per_head", "floor_per_head", "n_buckets",
-                 "bucket_override", "head_w_per_unit", "sens_per_unit")]
+                 "bucket_override", "head_w_per_unit", "sens_per_unit", "value_norm")] + [("value_norm_eps", C.c_float)]
 
 
 @dataclass
@@ -60,6 +60,8 @@ class Problem:
     bucket_override: int = -1
     head_w_per_unit: bool = True
     sens_per_unit: bool = False
+    value_norm: bool = False          # Eq. 4's value-norm ratio rho on (True) or off (the "u = alpha" ablation)
+    value_norm_eps: float = 1e-6      # the eps of Alg. 1 (B)
 
     @property
     def n(self) -> int:
@@ -76,7 +78,7 @@ class Problem:
     def _params(self) -> _Params:
         return _Params(self.pool_kind, self.pool_size, self.budget_per_head, self.floor_per_head,
                        self.n_buckets, self.bucket_override, int(self.head_w_per_unit),
-                       int(self.sens_per_unit))
+                       int(self.sens_per_unit), int(self.value_norm), float(self.value_norm_eps))
 
 
 _lib = None
@@ -132,15 +134,33 @@ def pool1d(kind: int, size: int, x: np.ndarray) -> np.ndarray:
     return out
 
 
-def score(prob: Problem, q, k, head_w, want_csum: bool = False):
-    """(scores [Nu,Hkv,n], colmass [Nu,L][, csum [Nu,H,L]]) in fp64 (O1-O6)."""
+def vnorm(prob: Problem, v, eps: float | None = None) -> np.ndarray:
+    """rho [Nu,Hkv,L] in fp64: value-row norms over their mean plus eps (O5b)."""
+    v = _inp(v, prob)
+    rho = np.empty((prob.n_units, prob.n_kv_heads, prob.seq_len), np.float64)
+    s = prob._shape()
+    fn = lib().oracle_vnorm
+    fn.argtypes = [C.c_void_p, C.c_void_p, C.c_double, C.c_void_p]
+    # the parameter block carries eps as fp32
+    _check(fn(C.byref(s), _p(v), float(np.float32(prob.value_norm_eps)) if eps is None else float(eps), _p(rho)), "vnorm")
+    return rho
+
+
+def score(prob: Problem, q, k, head_w, want_csum: bool = False, v=None):
+    """(scores [Nu,Hkv,n], colmass [Nu,L][, csum [Nu,H,L]]) in fp64 (O1-O6); with prob.value_norm the values
+    `v` are needed for O5b."""
     q, k = _inp(q, prob), _inp(k, prob)
     head_w = np.ascontiguousarray(head_w, np.float32)
+    rho = None
+    if prob.value_norm:
+        if v is None:
+            raise ValueError("value_norm needs the values")
+        rho = vnorm(prob, v)
     scores = np.empty((prob.n_units, prob.n_kv_heads, prob.n), np.float64)
     colmass = np.empty((prob.n_units, prob.seq_len), np.float64)
     csum = np.empty((prob.n_units, prob.n_q_heads, prob.seq_len), np.float64) if want_csum else None
     s, p = prob._shape(), prob._params()
-    _check(lib().oracle_score(C.byref(s), C.byref(p), _p(q), _p(k), _p(head_w), _p(scores), _p(colmass),
+    _check(lib().oracle_score(C.byref(s), C.byref(p), _p(q), _p(k), _p(head_w), _p(rho), _p(scores), _p(colmass),
                               _p(csum)), "score")
     return (scores, colmass, csum) if want_csum else (scores, colmass)
 

@@ -18,7 +18,9 @@
  *   O3  column sum c_h[t] = sum_{i in Omega} A[h,i,t]           (Eq. 4, Alg. 1 (A))
  *   O4  scale      alpha_h[t] = (L / W) c_h[t]                          (Eq. 4)
  *   O5  1-D pooling of alpha_h over the prefix (argument; size 1 = the paper)
- *   O6  head table u_g[t] = max_{h in group g} W_head[h] * pooled_h[t]  (Eq. 6)
+ *   O5b value-norm ratio (optional) rho_g[t] = |v_g[t]|_2 / (mean_k |v_g[k]|_2 + eps),
+ *       u_h[t] = pooled_h[t] * rho_g[t]                    (Eq. 4, Alg. 1 (B))
+ *   O6  head table u_g[t] = max_{h in group g} W_head[h] * u_h[t]       (Eq. 6)
  *   O7  risk coordinate: entropy of the normalised window mass, bucket,
  *       threshold tau = table[bucket]                    (Eq. 7 left, Alg. 1 (A),(D))
  *   O8  candidate counts under tau (Eq. 8's candidate set) -> per-head budgets
@@ -29,7 +31,8 @@
  * Pins (tests/test_oracle_*.py): the mass identity sum_t c_h[t] = W (text after
  * Eq. 4), closed-form attention on constant / single-spike inputs, torch's fp64
  * softmax and pooling routines on special cases, Shannon entropy of uniform and
- * one-hot distributions, brute-force rational water-filling for O8, brute-force
+ * one-hot distributions, hand-computed norms, the mean identity and scale
+ * invariance of O5b, brute-force rational water-filling for O8, brute-force
  * sorting for O9, direct indexing for O10, FullKV reproduction, and the
  * identity |p - p~|_1 = 2m of Eq. A2.
  * Parity unpinned by the paper itself (the paper has no such step; pinned only
@@ -63,6 +66,8 @@ typedef struct {
   int32_t bucket_override; /* -1: bucket from the entropy */
   int32_t head_w_per_unit; /* 0: one [H] row shared by all units; 1: [Nu,H] */
   int32_t sens_per_unit;   /* 0: one [n_buckets] row; 1: [Nu,n_buckets] */
+  int32_t value_norm;      /* 1: multiply the pooled window mass by the value-norm ratio (O5b) */
+  float value_norm_eps;    /* the eps of Alg. 1 (B) */
 } or_params;
 
 /* exact widening of an input element to double */
@@ -165,12 +170,37 @@ int oracle_pool1d(int kind, int size, int n, const double *x, double *out) {
   return 0;
 }
 
+/* ------------------------------------------------------------------ O5b (Eq. 4's rho, Alg. 1 (B))
+ * r[t] = |v[u,g,t,:]|_2 over all L tokens, mu = mean_t r[t], rho[u,g,t] = r[t] / (mu + eps).
+ * Under GQA the values belong to the KV head, so the ratio is shared by the group's query heads. */
+int oracle_vnorm(const or_shape *s, const void *v, double eps, double *rho) {
+  const int L = s->seq_len, Hkv = s->n_kv_heads, Nu = s->n_units, d = s->head_dim;
+  for (int u = 0; u < Nu; ++u)
+    for (int g = 0; g < Hkv; ++g) {
+      double *r = rho + ((int64_t)u * Hkv + g) * (int64_t)L;
+      double total = 0.0;
+      for (int t = 0; t < L; ++t) {
+        double ss = 0.0;
+        for (int j = 0; j < d; ++j) {
+          const double x = widen(v, s->dtype, (((int64_t)u * Hkv + g) * L + t) * d + j);
+          ss += x * x;
+        }
+        r[t] = sqrt(ss);
+        total += r[t];
+      }
+      const double mu = total / (double)L;
+      for (int t = 0; t < L; ++t) r[t] = r[t] / (mu + eps);
+    }
+  return 0;
+}
+
 /* ------------------------------------------------------------------ O4-O6 (+ the mass for O7)
- * scores  [Nu,Hkv,n] : u_g[t] = max_{h in g} head_w[h] * pool((L/W) c_h)[t]
+ * scores  [Nu,Hkv,n] : u_g[t] = max_{h in g} head_w[h] * (pool((L/W) c_h)[t] * rho_g[t])
  * colmass [Nu,L]     : sum_h c_h[t]   (all heads of the unit, window columns included)
- * csum    [Nu,H,L]   : c_h[t] (optional) */
+ * csum    [Nu,H,L]   : c_h[t] (optional)
+ * rho     [Nu,Hkv,L] : value-norm ratios of O5b, or NULL for rho = 1 (the paper's "u = alpha" ablation) */
 int oracle_score(const or_shape *s, const or_params *p, const void *q, const void *k, const float *head_w,
-                 double *scores, double *colmass, double *csum_or_null) {
+                 const double *rho_or_null, double *scores, double *colmass, double *csum_or_null) {
   const int L = s->seq_len, W = s->window, H = s->n_q_heads, Hkv = s->n_kv_heads, Nu = s->n_units;
   if (H % Hkv || W > L || W < 1) return 1;
   const int G = H / Hkv, n = L - W;
@@ -196,7 +226,8 @@ int oracle_score(const or_shape *s, const or_params *p, const void *q, const voi
         for (int t = 0; t < n; ++t) alpha[t] = ((double)L / (double)W) * c[t];
         oracle_pool1d(p->pool_kind, p->pool_size, n, alpha, pooled);
         for (int t = 0; t < n; ++t) {
-          const double v = w * pooled[t];
+          const double ratio = rho_or_null ? rho_or_null[((int64_t)u * Hkv + g) * (int64_t)L + t] : 1.0;
+          const double v = w * (pooled[t] * ratio);
           if (v > out[t]) out[t] = v;
         }
       }
@@ -438,15 +469,18 @@ int oracle_compress(const or_shape *s, const or_params *p, const void *q, const 
   const int L = s->seq_len, W = s->window, Hkv = s->n_kv_heads, Nu = s->n_units, n = L - W;
   double *scores = scores_or_null ? scores_or_null : (double *)malloc(sizeof(double) * (size_t)Nu * Hkv * (n > 0 ? n : 1));
   double *colmass = (double *)malloc(sizeof(double) * (size_t)Nu * L);
+  double *rho = p->value_norm ? (double *)malloc(sizeof(double) * (size_t)Nu * Hkv * L) : NULL;
   int rc = 2;
-  if (scores && colmass) {
-    rc = oracle_score(s, p, q, k, head_w, scores, colmass, NULL);
+  if (scores && colmass && (rho || !p->value_norm)) {
+    rc = rho ? oracle_vnorm(s, v, (double)p->value_norm_eps, rho) : 0;
+    if (!rc) rc = oracle_score(s, p, q, k, head_w, rho, scores, colmass, NULL);
     if (!rc) rc = oracle_budget(s, p, scores, colmass, sens, budgets, offsets, bucket, entropy, NULL, NULL);
     if (!rc) rc = oracle_select(s, scores, budgets, offsets, indices);
     if (!rc) rc = oracle_gather(s, k, v, indices, budgets, offsets, k_out, v_out);
   }
   if (!scores_or_null) free(scores);
   free(colmass);
+  free(rho);
   return rc;
 }
 

@@ -413,3 +413,59 @@ def test_operating_points_from_the_paper():
     c2, c4 = gen.CONFIGS["c2"], gen.CONFIGS["c4"]
     assert (str(c2.seq_len), str(c2.budget_per_head), "1.56") in [tuple(r) for r in rows]
     assert (str(c4.seq_len), str(c4.budget_per_head), "-") in [tuple(r) for r in rows]
+
+
+# ---------------------------------------------------------------------------- O5b: value-norm ratio (Eq. 4)
+def test_vnorm_hand_example():
+    """Rows of norms 5, 0, 10, 1 (3-4-5 triangles): mean 4, so rho = 1.25, 0, 2.5, 0.25; with eps = 1 the
+    denominator is 5 (Alg. 1 (B): r / (mu + eps))."""
+    v = np.zeros((1, 1, 4, 8), np.float32)
+    v[0, 0, 0, :2] = (3, 4)
+    v[0, 0, 2, 3:5] = (6, 8)
+    v[0, 0, 3, 7] = -1
+    prob = Problem(1, 1, 1, 4, 1, head_dim=8, dtype=oracle.F32)
+    np.testing.assert_allclose(oracle.vnorm(prob, v, eps=0.0)[0, 0], [1.25, 0.0, 2.5, 0.25], rtol=1e-15)
+    np.testing.assert_allclose(oracle.vnorm(prob, v, eps=1.0)[0, 0], [1.0, 0.0, 2.0, 0.2], rtol=1e-15)
+
+
+@pytest.mark.parametrize("dtype", [oracle.F32, oracle.BF16])
+def test_vnorm_identities_and_library_norm(dtype):
+    """mean_t rho = mu / (mu + eps) (Eq. 4 divides by the mean); eps = 0 makes rho invariant to the scale of V
+    (the point of the 'head-relative normalisation'); rows of equal norm all get mu / (mu + eps); and the norms
+    agree with torch.linalg.vector_norm on the exactly widened inputs."""
+    prob, _, _, v = rand_case(11, Nu=2, H=4, Hkv=2, L=70, W=6, d=16, dtype=dtype)
+    vn = gen.as_numpy(v)
+    r = torch.linalg.vector_norm(v.double(), dim=-1).numpy()              # [Nu,Hkv,L]
+    mu = r.mean(-1, keepdims=True)
+    for eps in (0.0, 1e-6, 0.5):
+        rho = oracle.vnorm(prob, vn, eps=eps)
+        np.testing.assert_allclose(rho, r / (mu + eps), rtol=1e-13)
+        np.testing.assert_allclose(rho.mean(-1), (mu / (mu + eps))[..., 0], rtol=1e-13)
+    if dtype == oracle.F32:
+        np.testing.assert_allclose(oracle.vnorm(prob, 4.0 * vn, eps=0.0), oracle.vnorm(prob, vn, eps=0.0), rtol=1e-13)
+        unit = vn / np.linalg.norm(vn, axis=-1, keepdims=True) * 3.0        # every row has norm 3 (to fp32 rounding)
+        np.testing.assert_allclose(oracle.vnorm(prob, unit.astype(np.float32), eps=1.0), 0.75, rtol=1e-6)
+
+
+@pytest.mark.parametrize("pool_kind,pool_size", [(oracle.POOL_NONE, 1), (oracle.POOL_MAX, 5), (oracle.POOL_AVG, 3)])
+def test_score_applies_the_value_norm_after_pooling_and_before_the_head_max(pool_kind, pool_size):
+    """u_h = pool(alpha_h) * rho_g (Eq. 4; the pooling smooths the attention mass only), then Eq. 6's weighted
+    max over the group.  rho is shared by a group's heads and non-negative, so the score equals rho times the
+    score without it -- which pooling alpha * rho instead would break -- and the column mass does not change."""
+    prob, q, k, v = rand_case(5, Nu=2, H=4, Hkv=2, L=80, W=8, d=16)
+    v[:, :, 10] *= 25.0                                                    # one loud value row per head
+    prob.pool_kind, prob.pool_size = pool_kind, pool_size
+    qn, kn, vn = gen.as_numpy(q), gen.as_numpy(k), gen.as_numpy(v)
+    w = (0.5 + torch.rand(2, 4, generator=torch.Generator().manual_seed(1))).numpy().astype(np.float32)
+    plain, cm0 = oracle.score(prob, qn, kn, w)
+    prob.value_norm, prob.value_norm_eps = True, 1e-3
+    rho = oracle.vnorm(prob, vn)
+    with_rho, cm1 = oracle.score(prob, qn, kn, w, v=vn)
+    np.testing.assert_allclose(with_rho, plain * rho[:, :, :prob.n], rtol=1e-13)
+    np.testing.assert_array_equal(cm0, cm1)
+    if pool_size > 1:      # the other order of the two steps gives something else next to the loud row
+        assert not np.allclose(with_rho[:, :, 9], (plain * rho[:, :, :prob.n])[:, :, 10])
+    # the whole pass uses the same scores
+    prob.budget_per_head = 24
+    out = oracle.compress(prob, qn, kn, vn, w, gen.as_numpy(gen.make_sens(gen.CONFIGS["c1"])))
+    np.testing.assert_array_equal(out["scores"], with_rho)
