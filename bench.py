@@ -164,6 +164,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2", choices=sorted(gen.CONFIGS))
     ap.add_argument("--units", type=int, default=0, help="units per GPU (default: the workload's)")
+    ap.add_argument("--value-norm", action="store_true",
+                    help="also apply Eq. 4's value-norm ratio (streams V once more; not the headline configuration)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -195,7 +197,7 @@ def main():
     units = [rank * n_units + u for u in range(n_units)]
     batch = gen.make_batch(cfg, dev, units)
     P = B.Params(pool_kind=cfg.pool_kind, pool_size=cfg.pool_size, budget_per_head=cfg.budget_per_head,
-                 floor_per_head=cfg.floor_per_head, n_buckets=cfg.n_buckets)
+                 floor_per_head=cfg.floor_per_head, n_buckets=cfg.n_buckets, value_norm=args.value_norm)
     shape = B.make_shape(batch["q"], batch["k"])
     params = B.make_params(P, batch["head_w"], batch["sens"])
     ws = B.alloc_workspace(shape, params, dev)
@@ -261,9 +263,21 @@ def main():
     torch.cuda.synchronize()
     stage_ms = {nm: sum(evs[it][j].elapsed_time(evs[it][j + 1]) for it in range(args.steps)) / args.steps
                 for j, nm in enumerate(stage_names)}
+    if args.value_norm:   # the extra stage, timed alone: V streamed once, scores rescaled
+        rho = torch.empty(n_units, Hkv, L, device=dev)
+        va, vb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        B.ckv_vnorm(shape, params, batch["v"], rho, scores, ws)
+        va.record()
+        for _ in range(args.steps):
+            B.ckv_vnorm(shape, params, batch["v"], rho, scores, ws)
+        vb.record()
+        torch.cuda.synchronize()
+        stage_ms["value_norm"] = va.elapsed_time(vb) / args.steps
 
     peak, peak_kind = measured_peaks()
     k2_bytes, gather_bytes = algorithmic_bytes(cfg, n_units)
+    if args.value_norm:
+        gather_bytes += k2_bytes // 2     # V read once: as many bytes as one pass over K
     scan_gbs = k2_bytes / (scan_ms * 1e-3) / 1e9
     traffic = SCAN_DRAM_TRAFFIC_PER_UNIT.get(cfg.name)
     traffic = traffic * n_units if traffic is not None else None
@@ -325,7 +339,8 @@ def main():
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if cfg.dtype == "bf16" else "f32",
-                "data": "synthetic", "config": config_dict(cfg, n_units, world), "clocks": clocks, "e2e": e2e,
+                "data": "synthetic", "config": dict(config_dict(cfg, n_units, world), **({"value_norm": True} if args.value_norm else {})),
+                "clocks": clocks, "e2e": e2e,
                 "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu_baseline}
         print(json.dumps(line), flush=True)
     if world > 1:

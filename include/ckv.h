@@ -71,6 +71,9 @@ typedef struct {
   int32_t bucket_override;  /* -1: bucket from the entropy of the unit's window mass; else that bucket */
   int64_t head_w_stride_unit; /* elements between the head_w rows of consecutive units; 0 = one row for all */
   int64_t sens_stride_unit;   /* same for the threshold table */
+  int32_t value_norm;       /* 1: ckv_compress multiplies the scores by the value-norm ratio rho of Eq. 4
+                               (see ckv_vnorm); 0: u = alpha, the paper's ablation without it */
+  float value_norm_eps;     /* the eps of Alg. 1 (B), >= 0 */
 } ckv_params;
 
 /* Bytes of work space any entry point needs for this problem (0 on invalid arguments). */
@@ -108,6 +111,18 @@ ckv_status ckv_score(const ckv_shape* shape, const ckv_params* params, const voi
 ckv_status ckv_budget(const ckv_shape* shape, const ckv_params* params, const float* scores,
                       const float* colmass, const float* sens, int32_t* budgets, int32_t* offsets,
                       int32_t* bucket, float* entropy, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Value-norm ratio of the stabilised utility (Eq. 4, Alg. 1 (B)), per unit and KV head (under GQA the
+ * values belong to the KV head, so a group's query heads share it):
+ *   r[t] = |v[t,:]|_2 over all L tokens;  rho[t] = r[t] / (mean_t r[t] + value_norm_eps)
+ * rho [Nu,Hkv,L] fp32 (output).  When scores_or_null [Nu,Hkv,n] is given, scores[g,t] *= rho[g,t] in
+ * place for the prefix: Eq. 4's u = alpha * rho applied after the pooling and, because rho >= 0 is
+ * common to the group, equal to applying it before Eq. 6's maximum.  v is read once (Hkv L d elements
+ * per unit).  Runs whatever params->value_norm says; that flag only steers ckv_compress.
+ */
+ckv_status ckv_vnorm(const ckv_shape* shape, const ckv_params* params, const void* v, float* rho,
+                     float* scores_or_null, void* ws, size_t ws_bytes, void* stream);
 
 /*
  * Per-head Top-k (Eq. 8's Top-B branch).  For every unit and KV head g the budgets[g] - W

@@ -16,7 +16,7 @@ void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
 static size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 
-WsLayout ws_layout(const ckv_shape& s, const ckv_params&) {
+WsLayout ws_layout(const ckv_shape& s, const ckv_params& p) {
   WsLayout w{};
   const size_t Nu = s.n_units, H = s.n_q_heads, Hkv = s.n_kv_heads, L = s.seq_len, W = s.window;
   const size_t n = L - W;
@@ -36,6 +36,8 @@ WsLayout ws_layout(const ckv_shape& s, const ckv_params&) {
     w.cnt_part = o, o = align_up(o + b.cnt_bytes);
     w.bud_done = o, o = align_up(o + b.done_bytes);
   }
+  w.vn_part = o, o = align_up(o + Nu * Hkv * ((L + kVnormRows - 1) / kVnormRows) * sizeof(float));
+  w.vn_rho = o, o = align_up(o + (p.value_norm ? Nu * Hkv * L * sizeof(float) : 0));
   if (s.dtype == CKV_BF16) {
     const TcLayout t = tc_layout(s);
     w.tc_part = o, o = align_up(o + t.part_bytes);
@@ -74,6 +76,8 @@ static ckv_status check_params(const ckv_shape* s, const ckv_params* p) {
   if (p->budget_per_head < 1 || p->floor_per_head < 0 || p->n_buckets < 1) return CKV_ERR_INVALID_ARG;
   if (p->bucket_override < -1 || p->bucket_override >= p->n_buckets) return CKV_ERR_INVALID_ARG;
   if (p->head_w_stride_unit < 0 || p->sens_stride_unit < 0) return CKV_ERR_INVALID_ARG;
+  if (p->value_norm != 0 && p->value_norm != 1) return CKV_ERR_INVALID_ARG;
+  if (!(p->value_norm_eps >= 0.f) || !(p->value_norm_eps < 3.0e38f)) return CKV_ERR_INVALID_ARG;
   if (p->budget_per_head < s->seq_len) {
     if (p->budget_per_head < s->window) return CKV_ERR_INVALID_ARG;
     if (p->floor_per_head > p->budget_per_head - s->window) return CKV_ERR_INVALID_ARG;
@@ -173,6 +177,20 @@ ckv_status ckv_budget(const ckv_shape* shape, const ckv_params* params, const fl
   return CKV_OK;
 }
 
+ckv_status ckv_vnorm(const ckv_shape* shape, const ckv_params* params, const void* v, float* rho,
+                     float* scores_or_null, void* ws, size_t ws_bytes, void* stream) {
+  CKV_TRY(check_shape(shape));
+  CKV_TRY(check_params(shape, params));
+  if (!all_aligned16({v}) || !all_aligned4({rho})) return CKV_ERR_INVALID_ARG;
+  if (scores_or_null && !aligned(scores_or_null, 4)) return CKV_ERR_INVALID_ARG;
+  CKV_TRY(check_ws(shape, params, ws, ws_bytes));
+  const WsLayout w = ws_layout(*shape, *params);
+  float* part = reinterpret_cast<float*>((char*)ws + w.vn_part);
+  CKV_CUDA(launch_vnorm_rows(*shape, v, rho, part, (cudaStream_t)stream));
+  CKV_CUDA(launch_vnorm_finish(*shape, params->value_norm_eps, rho, part, scores_or_null, (cudaStream_t)stream));
+  return CKV_OK;
+}
+
 ckv_status ckv_select(const ckv_shape* shape, const ckv_params* params, const float* scores, const int32_t* budgets,
                       const int32_t* offsets, int32_t* indices, void* ws, size_t ws_bytes, void* stream) {
   CKV_TRY(check_shape(shape));
@@ -212,6 +230,12 @@ ckv_status ckv_compress(const ckv_shape* shape, const ckv_params* params, const 
   int32_t* bucket = bucket_or_null ? bucket_or_null : reinterpret_cast<int32_t*>(base + w.bucket);
   float* entropy = entropy_or_null ? entropy_or_null : reinterpret_cast<float*>(base + w.entropy);
   CKV_TRY(score_impl(*shape, *params, q_win, k, head_w, scores, colmass, base, st));
+  if (params->value_norm) {   // Eq. 4: u = alpha * rho, before the thresholds see the scores
+    float* rho = reinterpret_cast<float*>(base + w.vn_rho);
+    float* part = reinterpret_cast<float*>(base + w.vn_part);
+    CKV_CUDA(launch_vnorm_rows(*shape, v, rho, part, st));
+    CKV_CUDA(launch_vnorm_finish(*shape, params->value_norm_eps, rho, part, scores, st));
+  }
   CKV_CUDA(launch_budget(*shape, *params, scores, sens, budgets, offsets, bucket, entropy, base + w.ent_part,
                          base + w.cnt_part, base + w.bud_done, st));
   CKV_CUDA(launch_select(*shape, *params, scores, budgets, offsets, indices, st));

@@ -12,6 +12,7 @@ constexpr int kMaxWindow = 64;
 constexpr int kMaxKvHeads = 64;
 constexpr int kPlainKeysPerBlock = 256;  // keys per CTA in the plain (SIMT) score kernels
 constexpr int kEntSpan = 512;            // positions per entropy partial of the budget stage
+constexpr int kVnormRows = 256;          // value rows per block sum of the value-norm stage
 constexpr int kCountSpan = 8192;         // scores per counting CTA of the budget stage
 
 // log2(e): the softmax is evaluated in base 2, x = (q.k) * log2(e) / sqrt(d)
@@ -33,6 +34,8 @@ struct WsLayout {
   size_t ent_part; // double [Nu, nblk]        entropy partials of the budget stage (nblk = ceil(L / kEntSpan))
   size_t cnt_part; // int32 [Nu, Hkv, S]       candidate counts per slice
   size_t bud_done; // int32 [Nu]               CTAs of the unit that have finished counting
+  size_t vn_part;  // float [Nu, Hkv, ceil(L / kVnormRows)] block sums of the value-row norms
+  size_t vn_rho;   // float [Nu, Hkv, L]       value-norm ratios of the fused call (only with value_norm)
   size_t total;
   int nblk;
 };
@@ -87,6 +90,11 @@ cudaError_t launch_entropy_partials(const ckv_shape& s, const float* colmass, vo
 cudaError_t launch_budget(const ckv_shape& s, const ckv_params& p, const float* scores, const float* sens,
                           int32_t* budgets, int32_t* offsets, int32_t* bucket, float* entropy, void* ent_part,
                           void* cnt_part, void* done, cudaStream_t st);
+// Value-norm ratio (Eq. 4's rho): row norms and block sums of V, then the division by mean + eps (and the
+// multiplication of the prefix scores when given).
+cudaError_t launch_vnorm_rows(const ckv_shape& s, const void* v, float* rho, float* part, cudaStream_t st);
+cudaError_t launch_vnorm_finish(const ckv_shape& s, float eps, float* rho, const float* part, float* scores,
+                                cudaStream_t st);
 cudaError_t launch_select(const ckv_shape& s, const ckv_params& p, const float* scores, const int32_t* budgets,
                           const int32_t* offsets, int32_t* indices, cudaStream_t st);
 cudaError_t launch_gather(const ckv_shape& s, const ckv_params& p, const void* k, const void* v,
