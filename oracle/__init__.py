@@ -39,7 +39,8 @@ class _Shape(C.Structure):
 class _Params(C.Structure):
     _fields_ = [(n, C.c_int32) for n in
                 ("pool_kind", "pool_size", "budget_per_head", "floor_per_head", "n_buckets",
-                 "bucket_override", "head_w_per_unit", "sens_per_unit", "value_norm")] + [("value_norm_eps", C.c_float)]
+                 "bucket_override", "head_w_per_unit", "sens_per_unit", "value_norm")] + \
+               [("value_norm_eps", C.c_float), ("shared_elastic", C.c_int32)]
 
 
 @dataclass
@@ -62,6 +63,7 @@ class Problem:
     sens_per_unit: bool = False
     value_norm: bool = False          # Eq. 4's value-norm ratio rho on (True) or off (the "u = alpha" ablation)
     value_norm_eps: float = 1e-6      # the eps of Alg. 1 (B)
+    shared_elastic: bool = False      # the paper's own selection: one elastic set per unit (Eq. 6 over all heads, Eq. 8)
 
     @property
     def n(self) -> int:
@@ -78,7 +80,8 @@ class Problem:
     def _params(self) -> _Params:
         return _Params(self.pool_kind, self.pool_size, self.budget_per_head, self.floor_per_head,
                        self.n_buckets, self.bucket_override, int(self.head_w_per_unit),
-                       int(self.sens_per_unit), int(self.value_norm), float(self.value_norm_eps))
+                       int(self.sens_per_unit), int(self.value_norm), float(self.value_norm_eps),
+                       int(self.shared_elastic))
 
 
 _lib = None
@@ -198,7 +201,8 @@ def select(prob: Problem, scores, budgets, offsets) -> np.ndarray:
     offsets = np.ascontiguousarray(offsets, np.int32)
     idx = np.full((prob.n_units, prob.n_kv_heads * prob.rows_per_head), -1, np.int32)
     s = prob._shape()
-    _check(lib().oracle_select(C.byref(s), _p(scores), _p(budgets), _p(offsets), _p(idx)), "select")
+    _check(lib().oracle_select(C.byref(s), _p(scores), _p(budgets), _p(offsets), C.c_int64(idx.shape[1]), _p(idx)),
+           "select")
     return idx
 
 
@@ -211,8 +215,8 @@ def gather(prob: Problem, k, v, indices, budgets, offsets):
     shape = (prob.n_units, prob.n_kv_heads * prob.rows_per_head, prob.head_dim)
     ko, vo = np.zeros(shape, k.dtype), np.zeros(shape, v.dtype)
     s = prob._shape()
-    _check(lib().oracle_gather(C.byref(s), _p(k), _p(v), _p(indices), _p(budgets), _p(offsets), _p(ko), _p(vo)),
-           "gather")
+    _check(lib().oracle_gather(C.byref(s), _p(k), _p(v), _p(indices), _p(budgets), _p(offsets),
+                               C.c_int64(indices.shape[1]), _p(ko), _p(vo)), "gather")
     return ko, vo
 
 
@@ -240,9 +244,10 @@ def kept_mass(prob: Problem, q, k, indices, budgets, offsets) -> np.ndarray:
     q, k = _inp(q, prob), _inp(k, prob)
     kept = np.empty((prob.n_units, prob.n_q_heads, prob.window), np.float64)
     s = prob._shape()
-    _check(lib().oracle_kept_mass(C.byref(s), _p(q), _p(k), _p(np.ascontiguousarray(indices, np.int32)),
-                                  _p(np.ascontiguousarray(budgets, np.int32)),
-                                  _p(np.ascontiguousarray(offsets, np.int32)), _p(kept)), "kept_mass")
+    indices = np.ascontiguousarray(indices, np.int32)
+    _check(lib().oracle_kept_mass(C.byref(s), _p(q), _p(k), _p(indices), _p(np.ascontiguousarray(budgets, np.int32)),
+                                  _p(np.ascontiguousarray(offsets, np.int32)), C.c_int64(indices.shape[1]),
+                                  _p(kept)), "kept_mass")
     return kept
 
 

@@ -27,6 +27,9 @@
  *       clamped so that they sum to the total budget
  *   O9  Top-k per KV head, ties to the lowest index, window always kept (Eq. 8)
  *   O10 gather of the kept K/V rows                               (Sec. 3, Alg. 1 (D))
+ * With shared_elastic set, O6-O9 take the paper's own form instead: the weighted max of
+ * Eq. 6 runs over all H heads of the unit, the retained set is Eq. 8's (all candidates if
+ * they fit the budget, else the Top-B of them) and every KV head keeps that one set.
  *
  * Pins (tests/test_oracle_*.py): the mass identity sum_t c_h[t] = W (text after
  * Eq. 4), closed-form attention on constant / single-spike inputs, torch's fp64
@@ -68,6 +71,7 @@ typedef struct {
   int32_t sens_per_unit;   /* 0: one [n_buckets] row; 1: [Nu,n_buckets] */
   int32_t value_norm;      /* 1: multiply the pooled window mass by the value-norm ratio (O5b) */
   float value_norm_eps;    /* the eps of Alg. 1 (B) */
+  int32_t shared_elastic;  /* 1: one elastic set per unit (Eq. 6 over all heads, Eq. 8), shared by its KV heads */
 } or_params;
 
 /* exact widening of an input element to double */
@@ -232,6 +236,17 @@ int oracle_score(const or_shape *s, const or_params *p, const void *q, const voi
         }
       }
     }
+    if (p->shared_elastic) {
+      /* Eq. 6 over all H heads of the unit: the max of the groups' maxima; every KV head carries it */
+      for (int t = 0; t < n; ++t) {
+        double m = -INFINITY;
+        for (int g = 0; g < Hkv; ++g) {
+          const double x = scores[((int64_t)u * Hkv + g) * (int64_t)n + t];
+          if (x > m) m = x;
+        }
+        for (int g = 0; g < Hkv; ++g) scores[((int64_t)u * Hkv + g) * (int64_t)n + t] = m;
+      }
+    }
     free(alpha);
     free(pooled);
   }
@@ -375,6 +390,16 @@ int oracle_budget(const or_shape *s, const or_params *p, const double *scores, c
     }
     if (B >= L) {
       for (int g = 0; g < Hkv; ++g) e[g] = n; /* FullKV: the whole prefix, then the window */
+    } else if (p->shared_elastic) {
+      /* Eq. 8: all candidates when they fit the budget, else the Top-B of them (B counts the window here);
+       * the floor argument still bounds the prefix part from below.  The heads' scores are identical. */
+      const double *sc = scores + (int64_t)u * Hkv * (int64_t)n;
+      int64_t c = 0;
+      for (int t = 0; t < n; ++t) c += (sc[t] >= tau);
+      int64_t keep = c < (int64_t)(B - W) ? c : (int64_t)(B - W);
+      if (keep < f) keep = f;
+      if (keep > n) keep = n;
+      for (int g = 0; g < Hkv; ++g) e[g] = keep;
     } else {
       int rc = oracle_allocate(Hkv, n, f, (int64_t)Hkv * (B - W), dem, e);
       if (rc) return 10 + rc;
@@ -407,18 +432,18 @@ static int by_index(const void *a, const void *b) {
   return (x->idx > y->idx) - (x->idx < y->idx);
 }
 
-/* indices [Nu, sum_g budgets] packed at offsets: per KV head the budgets[g] - W
- * best prefix positions in ascending order, then n .. L-1. */
+/* indices [Nu, unit_rows]: unit u starts at u * unit_rows (unit_rows = Hkv min(B, L), which the
+ * heads' budgets fill exactly unless the selection is elastic), head g at offsets[u,g]: the
+ * budgets[g] - W best prefix positions in ascending order, then n .. L-1. */
 int oracle_select(const or_shape *s, const double *scores, const int32_t *budgets, const int32_t *offsets,
-                  int32_t *indices) {
+                  int64_t unit_rows, int32_t *indices) {
   const int L = s->seq_len, W = s->window, Hkv = s->n_kv_heads, Nu = s->n_units, n = L - W;
   int err = 0;
 #pragma omp parallel for collapse(2) schedule(dynamic)
   for (int u = 0; u < Nu; ++u)
     for (int g = 0; g < Hkv; ++g) {
       const int e = budgets[(int64_t)u * Hkv + g] - W;
-      const int64_t rows_per_unit = offsets[(int64_t)u * (Hkv + 1) + Hkv];
-      int32_t *out = indices + (int64_t)u * rows_per_unit + offsets[(int64_t)u * (Hkv + 1) + g];
+      int32_t *out = indices + (int64_t)u * unit_rows + offsets[(int64_t)u * (Hkv + 1) + g];
       if (e < 0 || e > n) {
         err = 1;
         continue;
@@ -440,13 +465,12 @@ int oracle_select(const or_shape *s, const double *scores, const int32_t *budget
 
 /* ------------------------------------------------------------------ O10 */
 int oracle_gather(const or_shape *s, const void *k, const void *v, const int32_t *indices, const int32_t *budgets,
-                  const int32_t *offsets, void *k_out, void *v_out) {
+                  const int32_t *offsets, int64_t unit_rows, void *k_out, void *v_out) {
   const int L = s->seq_len, d = s->head_dim, Hkv = s->n_kv_heads, Nu = s->n_units;
   const size_t esz = s->dtype == OR_F32 ? 4 : 2, row = esz * (size_t)d;
   for (int u = 0; u < Nu; ++u) {
-    const int64_t rows_per_unit = offsets[(int64_t)u * (Hkv + 1) + Hkv];
     for (int g = 0; g < Hkv; ++g) {
-      const int64_t o = (int64_t)u * rows_per_unit + offsets[(int64_t)u * (Hkv + 1) + g];
+      const int64_t o = (int64_t)u * unit_rows + offsets[(int64_t)u * (Hkv + 1) + g];
       for (int j = 0; j < budgets[(int64_t)u * Hkv + g]; ++j) {
         const int32_t t = indices[o + j];
         if (t < 0 || t >= L) return 1;
@@ -475,8 +499,9 @@ int oracle_compress(const or_shape *s, const or_params *p, const void *q, const 
     rc = rho ? oracle_vnorm(s, v, (double)p->value_norm_eps, rho) : 0;
     if (!rc) rc = oracle_score(s, p, q, k, head_w, rho, scores, colmass, NULL);
     if (!rc) rc = oracle_budget(s, p, scores, colmass, sens, budgets, offsets, bucket, entropy, NULL, NULL);
-    if (!rc) rc = oracle_select(s, scores, budgets, offsets, indices);
-    if (!rc) rc = oracle_gather(s, k, v, indices, budgets, offsets, k_out, v_out);
+    const int64_t unit_rows = (int64_t)Hkv * (p->budget_per_head < L ? p->budget_per_head : L);
+    if (!rc) rc = oracle_select(s, scores, budgets, offsets, unit_rows, indices);
+    if (!rc) rc = oracle_gather(s, k, v, indices, budgets, offsets, unit_rows, k_out, v_out);
   }
   if (!scores_or_null) free(scores);
   free(colmass);
@@ -488,15 +513,14 @@ int oracle_compress(const or_shape *s, const or_params *p, const void *q, const 
  * kept[u,h,i] = sum_{t in S_g} A[h,i,t]: attention mass of window row i that
  * survives the selection; the discarded mass is m = 1 - kept. */
 int oracle_kept_mass(const or_shape *s, const void *q, const void *k, const int32_t *indices, const int32_t *budgets,
-                     const int32_t *offsets, double *kept) {
+                     const int32_t *offsets, int64_t unit_rows, double *kept) {
   const int L = s->seq_len, W = s->window, H = s->n_q_heads, Hkv = s->n_kv_heads, G = H / Hkv;
 #pragma omp parallel for collapse(2) schedule(dynamic)
   for (int u = 0; u < s->n_units; ++u)
     for (int h = 0; h < H; ++h) {
       const int g = h / G;
       double *row = (double *)malloc(sizeof(double) * (size_t)L);
-      const int64_t rows_per_unit = offsets[(int64_t)u * (Hkv + 1) + Hkv];
-      const int32_t *idx = indices + (int64_t)u * rows_per_unit + offsets[(int64_t)u * (Hkv + 1) + g];
+      const int32_t *idx = indices + (int64_t)u * unit_rows + offsets[(int64_t)u * (Hkv + 1) + g];
       for (int i = 0; i < W; ++i) {
         attention_row(s, q, k, u, h, i, row);
         double a = 0.0;

@@ -469,3 +469,74 @@ def test_score_applies_the_value_norm_after_pooling_and_before_the_head_max(pool
     prob.budget_per_head = 24
     out = oracle.compress(prob, qn, kn, vn, w, gen.as_numpy(gen.make_sens(gen.CONFIGS["c1"])))
     np.testing.assert_array_equal(out["scores"], with_rho)
+
+
+# ---------------------------------------------------------------------------- the paper's own selection (Eq. 6 over all heads, Eq. 8)
+def test_shared_elastic_selection_against_brute_force():
+    """shared_elastic: u^[t] = max over ALL heads of w_h * u_h[t] (Eq. 6), the set is Eq. 8's -- every candidate
+    when they fit the budget, else the Top-B of them -- and all KV heads keep it.  Built here from the per-head
+    mode's scores by numpy set operations and a stable sort."""
+    prob, q, k, v = rand_case(21, Nu=3, H=8, Hkv=4, L=120, W=8, d=16)
+    prob.pool_size, prob.budget_per_head, prob.floor_per_head = 1, 40, 0
+    qn, kn, vn = gen.as_numpy(q), gen.as_numpy(k), gen.as_numpy(v)
+    w = (0.5 + torch.rand(3, 8, generator=torch.Generator().manual_seed(2))).numpy().astype(np.float32)
+    per_head, cm = oracle.score(prob, qn, kn, w)
+    prob.shared_elastic = True
+    shared, cm2 = oracle.score(prob, qn, kn, w)
+    np.testing.assert_array_equal(shared, np.broadcast_to(per_head.max(1, keepdims=True), per_head.shape))
+    np.testing.assert_array_equal(cm, cm2)
+    u_hat = shared[:, 0]
+    n, W, B = prob.n, prob.window, prob.budget_per_head
+    # three thresholds: none, few (elastic under-retention) and many candidates (clamped to the budget)
+    for q_tau, regime in ((1.01, "none"), (0.9, "few"), (0.3, "many")):
+        tau = np.float32(np.quantile(u_hat, q_tau) if q_tau <= 1 else u_hat.max() * 2)
+        sens = np.full(prob.n_buckets, tau, np.float32)
+        bud = oracle.budget(prob, shared, cm, sens)
+        idx = oracle.select(prob, shared, bud["budgets"], bud["offsets"])
+        for u in range(3):
+            cand = np.nonzero(u_hat[u] >= np.float64(tau))[0]
+            if len(cand) <= B - W:
+                want = cand
+                assert regime in ("none", "few")
+            else:
+                order = np.argsort(-u_hat[u], kind="stable")         # ties to the lowest index
+                want = np.sort(order[:B - W])
+                assert regime == "many"
+            want = np.concatenate([want, np.arange(n, n + W)])
+            assert (bud["budgets"][u] == len(want)).all()
+            for g in range(4):
+                got = idx[u, bud["offsets"][u, g]: bud["offsets"][u, g + 1]]
+                np.testing.assert_array_equal(got, want)
+        if regime == "none":
+            assert (bud["budgets"] == W).all()
+    # the floor bounds the prefix part from below even with no candidate
+    prob.floor_per_head = 5
+    bud = oracle.budget(prob, shared, cm, np.full(prob.n_buckets, 1e9, np.float32))
+    assert (bud["budgets"] == W + 5).all()
+    # whole pass: every KV head gathers the same positions
+    prob.floor_per_head = 0
+    out = oracle.compress(prob, qn, kn, vn, w, np.full(prob.n_buckets, np.float32(np.quantile(u_hat, 0.9)), np.float32))
+    for u in range(3):
+        rows = out["budgets"][u, 0]
+        sets = [out["indices"][u, out["offsets"][u, g]: out["offsets"][u, g] + rows] for g in range(4)]
+        assert all((s == sets[0]).all() for s in sets)
+        for g in range(4):
+            np.testing.assert_array_equal(out["k_out"][u, out["offsets"][u, g]: out["offsets"][u, g] + rows],
+                                          kn[u, g, sets[0]])
+
+
+def test_shared_elastic_with_one_kv_head_and_a_full_pool_equals_the_per_head_mode():
+    """With a single KV head and more candidates than the budget both modes keep the Top-(B - W)."""
+    prob, q, k, v = rand_case(22, Nu=2, H=4, Hkv=1, L=90, W=6, d=16)
+    prob.budget_per_head, prob.floor_per_head = 30, 0
+    qn, kn = gen.as_numpy(q), gen.as_numpy(k)
+    w = np.ones((2, 4), np.float32)
+    sens = np.zeros(prob.n_buckets, np.float32)             # every position is a candidate
+    a_sc, a_cm = oracle.score(prob, qn, kn, w)
+    a = oracle.budget(prob, a_sc, a_cm, sens)
+    prob.shared_elastic = True
+    b_sc, b_cm = oracle.score(prob, qn, kn, w)
+    b = oracle.budget(prob, b_sc, b_cm, sens)
+    np.testing.assert_array_equal(a_sc, b_sc)
+    np.testing.assert_array_equal(a["budgets"], b["budgets"])
+    assert (b["budgets"] == 30).all()
