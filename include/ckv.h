@@ -74,6 +74,14 @@ typedef struct {
   int32_t value_norm;       /* 1: ckv_compress multiplies the scores by the value-norm ratio rho of Eq. 4
                                (see ckv_vnorm); 0: u = alpha, the paper's ablation without it */
   float value_norm_eps;     /* the eps of Alg. 1 (B), >= 0 */
+  int32_t shared_elastic;   /* 0: one index set per KV head, budgets clamped to sum to Hkv * B (the default);
+                               1: the paper's own selection -- Eq. 6's maximum over ALL heads of the unit, Eq. 8's
+                               elastic pool (every candidate if at most B - W of them, else the Top-(B - W)), one
+                               set shared by the unit's KV heads.  budgets[g] = W + kept are then equal for all g
+                               and may be smaller than B; rows of k_out, v_out, indices past offsets[u,Hkv] are
+                               left untouched.  ckv_compress applies it; staged callers run ckv_unit_max on the
+                               scores before ckv_budget. */
+  int32_t reserved_;        /* set to 0 */
 } ckv_params;
 
 /* Bytes of work space any entry point needs for this problem (0 on invalid arguments). */
@@ -125,10 +133,17 @@ ckv_status ckv_vnorm(const ckv_shape* shape, const ckv_params* params, const voi
                      float* scores_or_null, void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * Eq. 6 over all heads of a unit (used by the shared elastic selection): scores[u,g,t] is replaced, for
+ * every KV head g, by max_g' scores[u,g',t].  In place.
+ */
+ckv_status ckv_unit_max(const ckv_shape* shape, const ckv_params* params, float* scores, void* stream);
+
+/*
  * Per-head Top-k (Eq. 8's Top-B branch).  For every unit and KV head g the budgets[g] - W
  * largest of scores[g,0:n] are kept, equal scores resolved toward the lowest index; the kept
  * positions are written in ascending order and followed by the window n .. L-1, which is always
- * retained.  indices [Nu, Hkv * min(B,L)] int32, head g of unit u at row offsets[u,g].
+ * retained.  indices [Nu, Hkv * min(B,L)] int32, head g of unit u at row offsets[u,g] of the unit's
+ * Hkv * min(B,L) rows.
  */
 ckv_status ckv_select(const ckv_shape* shape, const ckv_params* params, const float* scores,
                       const int32_t* budgets, const int32_t* offsets, int32_t* indices, void* ws,

@@ -37,7 +37,8 @@ class ckv_params(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("pool_kind", "pool_size", "budget_per_head", "floor_per_head",
                                          "n_buckets", "bucket_override")] + \
                [(n, C.c_int64) for n in ("head_w_stride_unit", "sens_stride_unit")] + \
-               [("value_norm", C.c_int32), ("value_norm_eps", C.c_float)]
+               [("value_norm", C.c_int32), ("value_norm_eps", C.c_float), ("shared_elastic", C.c_int32),
+                ("reserved_", C.c_int32)]
 
 
 _lib = None
@@ -62,6 +63,7 @@ def lib() -> C.CDLL:
         L.ckv_budget.argtypes = [shp, prm, fp, fp, fp, i32p, i32p, i32p, fp, vp, sz, vp]
         L.ckv_select.argtypes = [shp, prm, fp, i32p, i32p, i32p, vp, sz, vp]
         L.ckv_vnorm.argtypes = [shp, prm, vp, fp, fp, vp, sz, vp]
+        L.ckv_unit_max.argtypes = [shp, prm, fp, vp]
         L.ckv_gather.argtypes = [shp, prm, vp, vp, i32p, i32p, vp, vp, vp]
         L.ckv_compress.argtypes = [shp, prm, vp, vp, vp, fp, fp, vp, vp, i32p, i32p, i32p, fp, i32p, fp, vp, sz, vp]
         L.ckv_compress_host.argtypes = [shp, prm, vp, vp, vp, fp, fp, vp, vp, i32p, i32p, i32p, vp, sz, vp, sz, vp]
@@ -74,7 +76,7 @@ def lib() -> C.CDLL:
         L.ckv_status_string.restype = C.c_char_p
         L.ckv_status_string.argtypes = [C.c_int]
         L.ckv_allocate_rows_host.argtypes = [C.c_int, C.c_int64, C.c_int64, C.c_int64, vp, vp]
-        for name in ("ckv_score", "ckv_score_noalloc", "ckv_budget", "ckv_select", "ckv_vnorm", "ckv_gather", "ckv_compress", "ckv_compress_host",
+        for name in ("ckv_score", "ckv_score_noalloc", "ckv_budget", "ckv_select", "ckv_vnorm", "ckv_unit_max", "ckv_gather", "ckv_compress", "ckv_compress_host",
                      "ckv_device_status", "ckv_version", "ckv_allocate_rows_host"):
             getattr(L, name).restype = C.c_int
         _lib = L
@@ -124,6 +126,7 @@ class Params:
     bucket_override: int = -1
     value_norm: bool = False
     value_norm_eps: float = 1e-6
+    shared_elastic: bool = False
 
 
 def _dtype_code(t: torch.Tensor) -> int:
@@ -148,7 +151,7 @@ def make_params(p: Params, head_w: torch.Tensor | None, sens: torch.Tensor | Non
     hw_stride = 0 if head_w is None or head_w.dim() == 1 else head_w.stride(0)
     se_stride = 0 if sens is None or sens.dim() == 1 else sens.stride(0)
     return ckv_params(p.pool_kind, p.pool_size, p.budget_per_head, p.floor_per_head, p.n_buckets,
-                      p.bucket_override, hw_stride, se_stride, int(p.value_norm), float(p.value_norm_eps))
+                      p.bucket_override, hw_stride, se_stride, int(p.value_norm), float(p.value_norm_eps), int(p.shared_elastic), 0)
 
 
 def _ptr(t):
@@ -208,6 +211,10 @@ def ckv_budget(shape, params, scores, colmass, sens, budgets, offsets, bucket, e
 def ckv_vnorm(shape, params, v, rho, scores, ws, stream=None):
     _check(lib().ckv_vnorm(C.byref(shape), C.byref(params), _ptr(v), _ptr(rho), _ptr(scores), _ptr(ws), ws.numel(),
                            _stream(stream)), "ckv_vnorm")
+
+
+def ckv_unit_max(shape, params, scores, stream=None):
+    _check(lib().ckv_unit_max(C.byref(shape), C.byref(params), _ptr(scores), _stream(stream)), "ckv_unit_max")
 
 
 def ckv_select(shape, params, scores, budgets, offsets, indices, ws, stream=None):

@@ -77,6 +77,7 @@ static ckv_status check_params(const ckv_shape* s, const ckv_params* p) {
   if (p->bucket_override < -1 || p->bucket_override >= p->n_buckets) return CKV_ERR_INVALID_ARG;
   if (p->head_w_stride_unit < 0 || p->sens_stride_unit < 0) return CKV_ERR_INVALID_ARG;
   if (p->value_norm != 0 && p->value_norm != 1) return CKV_ERR_INVALID_ARG;
+  if (p->shared_elastic != 0 && p->shared_elastic != 1) return CKV_ERR_INVALID_ARG;
   if (!(p->value_norm_eps >= 0.f) || !(p->value_norm_eps < 3.0e38f)) return CKV_ERR_INVALID_ARG;
   if (p->budget_per_head < s->seq_len) {
     if (p->budget_per_head < s->window) return CKV_ERR_INVALID_ARG;
@@ -191,6 +192,14 @@ ckv_status ckv_vnorm(const ckv_shape* shape, const ckv_params* params, const voi
   return CKV_OK;
 }
 
+ckv_status ckv_unit_max(const ckv_shape* shape, const ckv_params* params, float* scores, void* stream) {
+  CKV_TRY(check_shape(shape));
+  CKV_TRY(check_params(shape, params));
+  if (!all_aligned4({scores})) return CKV_ERR_INVALID_ARG;
+  CKV_CUDA(launch_unit_max(*shape, scores, (cudaStream_t)stream));
+  return CKV_OK;
+}
+
 ckv_status ckv_select(const ckv_shape* shape, const ckv_params* params, const float* scores, const int32_t* budgets,
                       const int32_t* offsets, int32_t* indices, void* ws, size_t ws_bytes, void* stream) {
   CKV_TRY(check_shape(shape));
@@ -236,6 +245,7 @@ ckv_status ckv_compress(const ckv_shape* shape, const ckv_params* params, const 
     CKV_CUDA(launch_vnorm_rows(*shape, v, rho, part, st));
     CKV_CUDA(launch_vnorm_finish(*shape, params->value_norm_eps, rho, part, scores, st));
   }
+  if (params->shared_elastic) CKV_CUDA(launch_unit_max(*shape, scores, st));
   CKV_CUDA(launch_budget(*shape, *params, scores, sens, budgets, offsets, bucket, entropy, base + w.ent_part,
                          base + w.cnt_part, base + w.bud_done, st));
   CKV_CUDA(launch_select(*shape, *params, scores, budgets, offsets, indices, st));

@@ -94,6 +94,7 @@ __global__ void __launch_bounds__(kThreads) count_allocate(ckv_shape s, ckv_para
   __shared__ int cnt_s;
   __shared__ int last_s;
   __shared__ long long dem_s[kMaxKvHeads], e_s[kMaxKvHeads];
+  __shared__ int raw_s;   // candidates of head 0 (the shared elastic selection gives every head the same scores)
   const int u = blockIdx.y, L = s.seq_len, W = s.window, n = L - W, Hkv = s.n_kv_heads;
   const int g = blockIdx.x / S, slice = blockIdx.x - g * S;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -145,11 +146,21 @@ __global__ void __launch_bounds__(kThreads) count_allocate(ckv_shape s, ckv_para
     int cc = 0;
     for (int sl = lane; sl < S; sl += 32) cc += __ldcg(cnt_part + ((int64_t)u * Hkv + gg) * S + sl);
     cc = __reduce_add_sync(0xffffffffu, cc);
-    if (lane == 0) dem_s[gg] = cc < lowest ? lowest : (cc > n ? n : cc);
+    if (lane == 0) {
+      dem_s[gg] = cc < lowest ? lowest : (cc > n ? n : cc);
+      if (gg == 0) raw_s = cc;
+    }
   }
   __syncthreads();
   if (B >= L) {
     if ((int)threadIdx.x < Hkv) e_s[threadIdx.x] = n;
+    __syncthreads();
+  } else if (p.shared_elastic) {
+    // Eq. 8: all candidates when they fit the budget, else the Top-B of them; the floor still applies
+    long long keep = raw_s < B - W ? raw_s : B - W;
+    keep = keep < f ? f : keep;
+    keep = keep > n ? n : keep;
+    if ((int)threadIdx.x < Hkv) e_s[threadIdx.x] = keep;
     __syncthreads();
   } else if (!allocate_rows_cta(Hkv, n, f, (long long)Hkv * (B - W), dem_s, e_s)) {
     if ((int)threadIdx.x < Hkv) e_s[threadIdx.x] = B - W;  // unreachable for validated arguments
@@ -169,7 +180,26 @@ __global__ void __launch_bounds__(kThreads) count_allocate(ckv_shape s, ckv_para
   if (entropy_out) entropy_out[u] = (float)ent_s;
 }
 
+// Eq. 6 over all heads of the unit: every KV head's score row becomes the maximum over the unit's rows.
+__global__ void __launch_bounds__(kThreads) unit_max_kernel(ckv_shape s, float* __restrict__ scores) {
+  const int u = blockIdx.y, Hkv = s.n_kv_heads, n = s.seq_len - s.window;
+  const int t = blockIdx.x * kThreads + threadIdx.x;
+  if (t >= n) return;
+  float* row = scores + (int64_t)u * Hkv * n + t;
+  float m = row[0];
+  for (int g = 1; g < Hkv; ++g) m = fmaxf(m, row[(int64_t)g * n]);
+  for (int g = 0; g < Hkv; ++g) row[(int64_t)g * n] = m;
+}
+
 }  // namespace
+
+cudaError_t launch_unit_max(const ckv_shape& s, float* scores, cudaStream_t st) {
+  const int n = s.seq_len - s.window;
+  if (n <= 0 || s.n_kv_heads < 2) return cudaSuccess;
+  unit_max_kernel<<<dim3((n + kThreads - 1) / kThreads, s.n_units), kThreads, 0, st>>>(s, scores);
+  count_launch();
+  return cudaGetLastError();
+}
 
 BudgetLayout budget_layout(const ckv_shape& s) {
   BudgetLayout b{};

@@ -95,6 +95,8 @@ cudaError_t launch_budget(const ckv_shape& s, const ckv_params& p, const float* 
 cudaError_t launch_vnorm_rows(const ckv_shape& s, const void* v, float* rho, float* part, cudaStream_t st);
 cudaError_t launch_vnorm_finish(const ckv_shape& s, float eps, float* rho, const float* part, float* scores,
                                 cudaStream_t st);
+// Eq. 6 over all heads of a unit (the shared elastic selection): scores[u,g,:] <- max_g' scores[u,g',:].
+cudaError_t launch_unit_max(const ckv_shape& s, float* scores, cudaStream_t st);
 cudaError_t launch_select(const ckv_shape& s, const ckv_params& p, const float* scores, const int32_t* budgets,
                           const int32_t* offsets, int32_t* indices, cudaStream_t st);
 cudaError_t launch_gather(const ckv_shape& s, const ckv_params& p, const void* k, const void* v,

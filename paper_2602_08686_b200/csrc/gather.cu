@@ -21,6 +21,7 @@ __global__ void __launch_bounds__(256) gather_kernel(ckv_shape s, int rows_per_h
     const int u = (int)(row / rows_per_unit);
     const int r = (int)(row - (int64_t)u * rows_per_unit);
     const int32_t* off = offsets + (int64_t)u * (Hkv + 1);
+    if (r >= off[Hkv]) continue;   // an elastic selection keeps fewer rows than the unit's share of the output
     int g = 0;
     while (g + 1 < Hkv && r >= off[g + 1]) ++g;
     const int t = indices[row];

@@ -57,7 +57,8 @@ __device__ __forceinline__ void transpose32(uint32_t (&a)[32]) {
 // Every warp then sends its counts to all CTAs of the cluster through distributed shared memory and the
 // step's barrier spans the cluster.
 template <int kCluster>
-__global__ void __launch_bounds__(kThreads) select_sliced_kernel(ckv_shape s, const float* __restrict__ scores,
+__global__ void __launch_bounds__(kThreads) select_sliced_kernel(ckv_shape s, int64_t unit_rows,
+                                                                 const float* __restrict__ scores,
                                                                  const int32_t* __restrict__ budgets,
                                                                  const int32_t* __restrict__ offsets,
                                                                  int32_t* __restrict__ indices) {
@@ -69,8 +70,7 @@ __global__ void __launch_bounds__(kThreads) select_sliced_kernel(ckv_shape s, co
   const int head = blockIdx.x / kCluster, rank = blockIdx.x % kCluster;
   const int u = head / Hkv, g = head % Hkv;
   const int e = budgets[(int64_t)u * Hkv + g] - W;
-  const int64_t rows_per_unit = offsets[(int64_t)u * (Hkv + 1) + Hkv];
-  int32_t* out = indices + (int64_t)u * rows_per_unit + offsets[(int64_t)u * (Hkv + 1) + g];
+  int32_t* out = indices + (int64_t)u * unit_rows + offsets[(int64_t)u * (Hkv + 1) + g];
   const float* sc = scores + ((int64_t)u * Hkv + g) * n;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int cbase = rank * kSlicedMax;                      // first position of this CTA
@@ -191,7 +191,8 @@ __global__ void __launch_bounds__(kThreads) select_sliced_kernel(ckv_shape s, co
   }
 }
 
-__global__ void __launch_bounds__(kThreads) select_digit_kernel(ckv_shape s, const float* __restrict__ scores,
+__global__ void __launch_bounds__(kThreads) select_digit_kernel(ckv_shape s, int64_t unit_rows,
+                                                                const float* __restrict__ scores,
                                                                 const int32_t* __restrict__ budgets,
                                                                 const int32_t* __restrict__ offsets,
                                                                 int32_t* __restrict__ indices) {
@@ -206,8 +207,7 @@ __global__ void __launch_bounds__(kThreads) select_digit_kernel(ckv_shape s, con
   const int Hkv = s.n_kv_heads, W = s.window, n = s.seq_len - W;
   const int u = blockIdx.x / Hkv, g = blockIdx.x % Hkv;
   const int e = budgets[(int64_t)u * Hkv + g] - W;
-  const int64_t rows_per_unit = offsets[(int64_t)u * (Hkv + 1) + Hkv];
-  int32_t* out = indices + (int64_t)u * rows_per_unit + offsets[(int64_t)u * (Hkv + 1) + g];
+  int32_t* out = indices + (int64_t)u * unit_rows + offsets[(int64_t)u * (Hkv + 1) + g];
   const float* sc = scores + ((int64_t)u * Hkv + g) * n;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
@@ -330,7 +330,7 @@ __global__ void __launch_bounds__(kThreads) select_digit_kernel(ckv_shape s, con
 
 
 template <int kCluster>
-cudaError_t launch_sliced(const ckv_shape& s, int n, const float* scores, const int32_t* budgets,
+cudaError_t launch_sliced(const ckv_shape& s, int n, int64_t unit_rows, const float* scores, const int32_t* budgets,
                           const int32_t* offsets, int32_t* indices, cudaStream_t st) {
   const int per_cta = (n + kCluster - 1) / kCluster;   // staging covers the fullest CTA
   const size_t smem = (size_t)((std::min(per_cta, kSlicedMax) + 1023) / 1024) * 1024 * sizeof(uint32_t);
@@ -346,21 +346,23 @@ cudaError_t launch_sliced(const ckv_shape& s, int n, const float* scores, const 
   attr.id = cudaLaunchAttributeClusterDimension;
   attr.val.clusterDim.x = kCluster, attr.val.clusterDim.y = 1, attr.val.clusterDim.z = 1;
   cfg.attrs = &attr, cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, select_sliced_kernel<kCluster>, s, scores, budgets, offsets, indices);
+  return cudaLaunchKernelEx(&cfg, select_sliced_kernel<kCluster>, s, unit_rows, scores, budgets, offsets, indices);
 }
 
 }  // namespace
 
-cudaError_t launch_select(const ckv_shape& s, const ckv_params&, const float* scores, const int32_t* budgets,
+cudaError_t launch_select(const ckv_shape& s, const ckv_params& p, const float* scores, const int32_t* budgets,
                           const int32_t* offsets, int32_t* indices, cudaStream_t st) {
   const int n = s.seq_len - s.window;
+  // unit u's indices start at u * unit_rows; its heads' budgets fill that exactly unless the selection is elastic
+  const int64_t unit_rows = (int64_t)s.n_kv_heads * (p.budget_per_head < s.seq_len ? p.budget_per_head : s.seq_len);
   cudaError_t e;
-  if (n <= kSlicedMax) e = launch_sliced<1>(s, n, scores, budgets, offsets, indices, st);
-  else if (n <= 2 * kSlicedMax) e = launch_sliced<2>(s, n, scores, budgets, offsets, indices, st);
-  else if (n <= 4 * kSlicedMax) e = launch_sliced<4>(s, n, scores, budgets, offsets, indices, st);
-  else if (n <= 8 * kSlicedMax) e = launch_sliced<8>(s, n, scores, budgets, offsets, indices, st);
+  if (n <= kSlicedMax) e = launch_sliced<1>(s, n, unit_rows, scores, budgets, offsets, indices, st);
+  else if (n <= 2 * kSlicedMax) e = launch_sliced<2>(s, n, unit_rows, scores, budgets, offsets, indices, st);
+  else if (n <= 4 * kSlicedMax) e = launch_sliced<4>(s, n, unit_rows, scores, budgets, offsets, indices, st);
+  else if (n <= 8 * kSlicedMax) e = launch_sliced<8>(s, n, unit_rows, scores, budgets, offsets, indices, st);
   else {
-    select_digit_kernel<<<s.n_units * s.n_kv_heads, kThreads, 0, st>>>(s, scores, budgets, offsets, indices);
+    select_digit_kernel<<<s.n_units * s.n_kv_heads, kThreads, 0, st>>>(s, unit_rows, scores, budgets, offsets, indices);
     e = cudaGetLastError();
   }
   count_launch();

@@ -43,11 +43,13 @@ def llama_shape(L=32768, W=32, Nu=2, H=32, Hkv=8, d=128, dtype=B.BF16):
 
 def default_params(**kw):
     base = dict(pool_kind=B.POOL_MAX, pool_size=7, budget_per_head=512, floor_per_head=1, n_buckets=16,
-                bucket_override=-1, head_w_stride_unit=32, sens_stride_unit=0, value_norm=0, value_norm_eps=1e-6)
+                bucket_override=-1, head_w_stride_unit=32, sens_stride_unit=0, value_norm=0, value_norm_eps=1e-6,
+                shared_elastic=0, reserved_=0)
     base.update(kw)
     return B.ckv_params(*[base[k] for k in ("pool_kind", "pool_size", "budget_per_head", "floor_per_head",
                                             "n_buckets", "bucket_override", "head_w_stride_unit",
-                                            "sens_stride_unit", "value_norm", "value_norm_eps")])
+                                            "sens_stride_unit", "value_norm", "value_norm_eps", "shared_elastic",
+                                            "reserved_")])
 
 
 def test_argument_errors_are_found_on_the_host():
@@ -70,6 +72,7 @@ def test_argument_errors_are_found_on_the_host():
     assert score(s, default_params(floor_per_head=500)) == B.ERR_INVALID_ARG      # f > B - W
     assert score(s, default_params(bucket_override=16)) == B.ERR_INVALID_ARG
     assert score(s, default_params(value_norm=2)) == B.ERR_INVALID_ARG
+    assert score(s, default_params(shared_elastic=3)) == B.ERR_INVALID_ARG
     assert score(s, default_params(value_norm_eps=-1.0)) == B.ERR_INVALID_ARG
     assert score(s, default_params(value_norm_eps=float("nan"))) == B.ERR_INVALID_ARG
     assert lib.ckv_vnorm(C.byref(s), C.byref(p), None, fake, None, fake, big, None) == B.ERR_INVALID_ARG
