@@ -40,7 +40,8 @@ class _Params(C.Structure):
     _fields_ = [(n, C.c_int32) for n in
                 ("pool_kind", "pool_size", "budget_per_head", "floor_per_head", "n_buckets",
                  "bucket_override", "head_w_per_unit", "sens_per_unit", "value_norm")] + \
-               [("value_norm_eps", C.c_float), ("shared_elastic", C.c_int32)]
+               [("value_norm_eps", C.c_float), ("shared_elastic", C.c_int32), ("global_alpha", C.c_int32),
+                ("units_per_prompt", C.c_int32)]
 
 
 @dataclass
@@ -64,6 +65,8 @@ class Problem:
     value_norm: bool = False          # Eq. 4's value-norm ratio rho on (True) or off (the "u = alpha" ablation)
     value_norm_eps: float = 1e-6      # the eps of Alg. 1 (B)
     shared_elastic: bool = False      # the paper's own selection: one elastic set per unit (Eq. 6 over all heads, Eq. 8)
+    global_alpha: bool = False        # Alg. 1 (A): alpha and the risk coordinate from the mean over the prompt's layers and heads
+    units_per_prompt: int = 1         # layers per prompt (consecutive units) for global_alpha
 
     @property
     def n(self) -> int:
@@ -81,7 +84,7 @@ class Problem:
         return _Params(self.pool_kind, self.pool_size, self.budget_per_head, self.floor_per_head,
                        self.n_buckets, self.bucket_override, int(self.head_w_per_unit),
                        int(self.sens_per_unit), int(self.value_norm), float(self.value_norm_eps),
-                       int(self.shared_elastic))
+                       int(self.shared_elastic), int(self.global_alpha), int(self.units_per_prompt))
 
 
 _lib = None

@@ -30,6 +30,9 @@
  * With shared_elastic set, O6-O9 take the paper's own form instead: the weighted max of
  * Eq. 6 runs over all H heads of the unit, the retained set is Eq. 8's (all candidates if
  * they fit the budget, else the Top-B of them) and every KV head keeps that one set.
+ * With global_alpha set, O4 and O7 take the paper's form: the attention is averaged over all
+ * layers and heads of the prompt before the window sum (Alg. 1 (A)), so one alpha and one risk
+ * coordinate serve all of the prompt's units (units_per_prompt consecutive units each).
  *
  * Pins (tests/test_oracle_*.py): the mass identity sum_t c_h[t] = W (text after
  * Eq. 4), closed-form attention on constant / single-spike inputs, torch's fp64
@@ -72,6 +75,8 @@ typedef struct {
   int32_t value_norm;      /* 1: multiply the pooled window mass by the value-norm ratio (O5b) */
   float value_norm_eps;    /* the eps of Alg. 1 (B) */
   int32_t shared_elastic;  /* 1: one elastic set per unit (Eq. 6 over all heads, Eq. 8), shared by its KV heads */
+  int32_t global_alpha;    /* 1: alpha from the mean attention over all layers and heads of the prompt */
+  int32_t units_per_prompt; /* layers of one prompt: units [s N, (s + 1) N) belong to prompt s (global_alpha) */
 } or_params;
 
 /* exact widening of an input element to double */
@@ -212,22 +217,39 @@ int oracle_score(const or_shape *s, const or_params *p, const void *q, const voi
   if (!csum) return 2;
   int rc = oracle_colsum(s, q, k, csum);
   if (rc) goto done;
-#pragma omp parallel for schedule(dynamic)
-  for (int u = 0; u < Nu; ++u) {
-    double *alpha = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
-    double *pooled = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
+  for (int u = 0; u < Nu; ++u)
     for (int t = 0; t < L; ++t) {
       double m = 0.0;
       for (int h = 0; h < H; ++h) m += csum[((int64_t)u * H + h) * L + t];
       colmass[(int64_t)u * L + t] = m;
     }
+  if (p->global_alpha) {
+    /* Alg. 1 (A): A-bar = mean over layers and heads of the prompt; its window column sums are the mean of the
+     * units' column masses over N H.  Every unit of the prompt then carries the prompt's mean mass. */
+    const int N = p->units_per_prompt;
+    if (N < 1 || Nu % N) {
+      rc = 3;
+      goto done;
+    }
+    for (int s0 = 0; s0 < Nu; s0 += N)
+      for (int t = 0; t < L; ++t) {
+        double m = 0.0;
+        for (int u = s0; u < s0 + N; ++u) m += colmass[(int64_t)u * L + t];
+        for (int u = s0; u < s0 + N; ++u) colmass[(int64_t)u * L + t] = m / (double)N;
+      }
+  }
+#pragma omp parallel for schedule(dynamic)
+  for (int u = 0; u < Nu; ++u) {
+    double *alpha = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
+    double *pooled = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
     for (int g = 0; g < Hkv; ++g) {
       double *out = scores + ((int64_t)u * Hkv + g) * (int64_t)n;
       for (int t = 0; t < n; ++t) out[t] = -INFINITY;
       for (int h = g * G; h < (g + 1) * G; ++h) {
         const double w = (double)head_w[p->head_w_per_unit ? (int64_t)u * H + h : h];
         const double *c = csum + ((int64_t)u * H + h) * (int64_t)L;
-        for (int t = 0; t < n; ++t) alpha[t] = ((double)L / (double)W) * c[t];
+        for (int t = 0; t < n; ++t)   /* Eq. 4's alpha: this head's window mass, or the prompt-wide mean per head */
+          alpha[t] = ((double)L / (double)W) * (p->global_alpha ? colmass[(int64_t)u * L + t] / (double)H : c[t]);
         oracle_pool1d(p->pool_kind, p->pool_size, n, alpha, pooled);
         for (int t = 0; t < n; ++t) {
           const double ratio = rho_or_null ? rho_or_null[((int64_t)u * Hkv + g) * (int64_t)L + t] : 1.0;

@@ -540,3 +540,58 @@ def test_shared_elastic_with_one_kv_head_and_a_full_pool_equals_the_per_head_mod
     np.testing.assert_array_equal(a_sc, b_sc)
     np.testing.assert_array_equal(a["budgets"], b["budgets"])
     assert (b["budgets"] == 30).all()
+
+
+# ---------------------------------------------------------------------------- prompt-global alpha (Alg. 1 (A))
+def test_global_alpha_identities():
+    """global_alpha: A-bar is the mean attention over all layers and heads of the prompt, so
+    (a) every unit of a prompt reports the same column mass, which sums to W H (each of the W H softmax rows of a
+        unit sums to one) -- the reason alpha has mean one over the L keys (text after Eq. 4);
+    (b) with unit weights, no pooling and no value norm, every head's score IS alpha = (L/W) mass / H;
+    (c) alpha does not depend on the order of the prompt's layers, nor on the other prompt's data;
+    (d) a prompt of one layer with one head gives the per-head mode's scores;
+    (e) the weights enter as Eq. 6's max inside the group: score = alpha * max_{h in g} w_h."""
+    prob, q, k, v = rand_case(31, Nu=4, H=4, Hkv=2, L=64, W=8, d=16)
+    prob.pool_kind, prob.pool_size = oracle.POOL_NONE, 1
+    qn, kn = gen.as_numpy(q), gen.as_numpy(k)
+    ones = np.ones((4, 4), np.float32)
+    per_head, cm_units = oracle.score(prob, qn, kn, ones)
+    prob.global_alpha, prob.units_per_prompt = True, 2
+    sc, cm = oracle.score(prob, qn, kn, ones)
+    L, W, H, n = 64, 8, 4, prob.n
+    np.testing.assert_allclose(cm.sum(-1), W * H, rtol=1e-12)                                  # (a)
+    np.testing.assert_array_equal(cm[0], cm[1])
+    np.testing.assert_array_equal(cm[2], cm[3])
+    np.testing.assert_allclose(cm[0], (cm_units[0] + cm_units[1]) / 2, rtol=1e-13)             # mean over the layers
+    alpha = (L / W) * cm / H
+    np.testing.assert_allclose(alpha.mean(-1), 1.0, rtol=1e-12)
+    for g in range(2):
+        np.testing.assert_allclose(sc[:, g], alpha[:, :n], rtol=1e-13)                         # (b)
+    perm = [1, 0, 2, 3]
+    sc_p, _ = oracle.score(prob, qn[perm], kn[perm], ones)
+    np.testing.assert_allclose(sc_p[0], sc[0], rtol=1e-13)                                     # (c)
+    np.testing.assert_array_equal(sc_p[2:], sc[2:])
+    w = (0.5 + torch.rand(4, 4, generator=torch.Generator().manual_seed(3))).numpy().astype(np.float32)
+    sc_w, _ = oracle.score(prob, qn, kn, w)
+    wmax = w.astype(np.float64).reshape(4, 2, 2).max(-1)
+    np.testing.assert_allclose(sc_w, alpha[:, None, :n] * wmax[:, :, None], rtol=1e-13)        # (e)
+    prob1, q1, k1, _ = rand_case(32, Nu=3, H=1, Hkv=1, L=40, W=4, d=16)
+    a, _ = oracle.score(prob1, gen.as_numpy(q1), gen.as_numpy(k1), np.ones((3, 1), np.float32))
+    prob1.global_alpha, prob1.units_per_prompt = True, 1
+    b, _ = oracle.score(prob1, gen.as_numpy(q1), gen.as_numpy(k1), np.ones((3, 1), np.float32))
+    np.testing.assert_allclose(a, b, rtol=1e-13)                                               # (d)
+
+
+def test_global_alpha_pools_alpha_and_shares_the_risk_coordinate():
+    """The pooling acts on the prompt's alpha (library max pooling), and the entropy bucket is one per prompt."""
+    prob, q, k, v = rand_case(33, Nu=4, H=4, Hkv=2, L=64, W=8, d=16)
+    prob.pool_kind, prob.pool_size = oracle.POOL_MAX, 5
+    prob.global_alpha, prob.units_per_prompt = True, 2
+    qn, kn = gen.as_numpy(q), gen.as_numpy(k)
+    sc, cm = oracle.score(prob, qn, kn, np.ones((4, 4), np.float32))
+    alpha = torch.from_numpy((64 / 8) * cm[:, :prob.n] / 4)
+    pooled = torch.nn.functional.max_pool1d(alpha[:, None], 5, 1, 2)[:, 0].numpy()
+    np.testing.assert_allclose(sc[:, 0], pooled, rtol=1e-13)
+    bud = oracle.budget(prob, sc, cm, gen.as_numpy(gen.make_sens(gen.CONFIGS["c1"])))
+    assert bud["bucket"][0] == bud["bucket"][1] and bud["bucket"][2] == bud["bucket"][3]
+    assert bud["entropy"][0] == bud["entropy"][1]
