@@ -81,6 +81,12 @@ typedef struct {
                                and may be smaller than B; rows of k_out, v_out, indices past offsets[u,Hkv] are
                                left untouched.  ckv_compress applies it; staged callers run ckv_unit_max on the
                                scores before ckv_budget. */
+  int32_t global_alpha;     /* 1: the paper's prompt-wide window mass (Alg. 1 (A)): the attention is averaged over all
+                               layers and heads of the prompt before the window sum, so alpha, and the entropy that picks
+                               the threshold, are one per prompt; see ckv_prompt_mass / ckv_global_scores.  0 (default):
+                               per query head of the unit */
+  int32_t units_per_prompt; /* with global_alpha: units [s N, (s+1) N) of the call belong to prompt s (its layers);
+                               N >= 1 divides n_units.  Ignored otherwise (0 allowed) */
   int32_t reserved_;        /* set to 0 */
 } ckv_params;
 
@@ -131,6 +137,24 @@ ckv_status ckv_budget(const ckv_shape* shape, const ckv_params* params, const fl
  */
 ckv_status ckv_vnorm(const ckv_shape* shape, const ckv_params* params, const void* v, float* rho,
                      float* scores_or_null, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Prompt-global window mass (Alg. 1 (A): A-bar = mean over layers and heads; alpha = (T/W) sum_{j in Omega} A-bar[j,:]),
+ * for params->global_alpha.  After ckv_score:
+ *   ckv_prompt_mass    pmass[s,t] = sum over the prompt's units in this call of colmass[u,t]; pmass [Nu/N, L] fp32.
+ *   ckv_global_scores  alpha_s = (L/W) pmass[s] / (units_total * H);
+ *                      scores[u,g,t] = (max_{h in g} head_w[u,h]) * pool(alpha_s)[t]  (alpha >= 0, so Eq. 6's maximum
+ *                      over the group is its largest weight), overwriting ckv_score's per-head scores;
+ *                      colmass[u,:] = pmass[s,:] / units_total, so that ckv_budget takes one entropy per prompt.
+ * units_total is the prompt's number of units on ALL devices (>= units_per_prompt): where a prompt's layers are
+ * spread over several GPUs, the caller adds the ranks' pmass arrays between the two calls (the method's one
+ * exchange step; paper_2602_08686_b200/sharding.py has the all-reduce).  ckv_compress runs both calls itself with
+ * units_total = units_per_prompt.  The value-norm ratio and the selection follow as usual.
+ */
+ckv_status ckv_prompt_mass(const ckv_shape* shape, const ckv_params* params, const float* colmass, float* pmass,
+                           void* stream);
+ckv_status ckv_global_scores(const ckv_shape* shape, const ckv_params* params, const float* head_w,
+                             const float* pmass, int32_t units_total, float* scores, float* colmass, void* stream);
 
 /*
  * Eq. 6 over all heads of a unit (used by the shared elastic selection): scores[u,g,t] is replaced, for

@@ -38,7 +38,7 @@ class ckv_params(C.Structure):
                                          "n_buckets", "bucket_override")] + \
                [(n, C.c_int64) for n in ("head_w_stride_unit", "sens_stride_unit")] + \
                [("value_norm", C.c_int32), ("value_norm_eps", C.c_float), ("shared_elastic", C.c_int32),
-                ("reserved_", C.c_int32)]
+                ("global_alpha", C.c_int32), ("units_per_prompt", C.c_int32), ("reserved_", C.c_int32)]
 
 
 _lib = None
@@ -64,6 +64,8 @@ def lib() -> C.CDLL:
         L.ckv_select.argtypes = [shp, prm, fp, i32p, i32p, i32p, vp, sz, vp]
         L.ckv_vnorm.argtypes = [shp, prm, vp, fp, fp, vp, sz, vp]
         L.ckv_unit_max.argtypes = [shp, prm, fp, vp]
+        L.ckv_prompt_mass.argtypes = [shp, prm, fp, fp, vp]
+        L.ckv_global_scores.argtypes = [shp, prm, fp, fp, C.c_int32, fp, fp, vp]
         L.ckv_gather.argtypes = [shp, prm, vp, vp, i32p, i32p, vp, vp, vp]
         L.ckv_compress.argtypes = [shp, prm, vp, vp, vp, fp, fp, vp, vp, i32p, i32p, i32p, fp, i32p, fp, vp, sz, vp]
         L.ckv_compress_host.argtypes = [shp, prm, vp, vp, vp, fp, fp, vp, vp, i32p, i32p, i32p, vp, sz, vp, sz, vp]
@@ -76,7 +78,7 @@ def lib() -> C.CDLL:
         L.ckv_status_string.restype = C.c_char_p
         L.ckv_status_string.argtypes = [C.c_int]
         L.ckv_allocate_rows_host.argtypes = [C.c_int, C.c_int64, C.c_int64, C.c_int64, vp, vp]
-        for name in ("ckv_score", "ckv_score_noalloc", "ckv_budget", "ckv_select", "ckv_vnorm", "ckv_unit_max", "ckv_gather", "ckv_compress", "ckv_compress_host",
+        for name in ("ckv_score", "ckv_score_noalloc", "ckv_budget", "ckv_select", "ckv_vnorm", "ckv_unit_max", "ckv_prompt_mass", "ckv_global_scores", "ckv_gather", "ckv_compress", "ckv_compress_host",
                      "ckv_device_status", "ckv_version", "ckv_allocate_rows_host"):
             getattr(L, name).restype = C.c_int
         _lib = L
@@ -127,6 +129,8 @@ class Params:
     value_norm: bool = False
     value_norm_eps: float = 1e-6
     shared_elastic: bool = False
+    global_alpha: bool = False
+    units_per_prompt: int = 1
 
 
 def _dtype_code(t: torch.Tensor) -> int:
@@ -151,7 +155,8 @@ def make_params(p: Params, head_w: torch.Tensor | None, sens: torch.Tensor | Non
     hw_stride = 0 if head_w is None or head_w.dim() == 1 else head_w.stride(0)
     se_stride = 0 if sens is None or sens.dim() == 1 else sens.stride(0)
     return ckv_params(p.pool_kind, p.pool_size, p.budget_per_head, p.floor_per_head, p.n_buckets,
-                      p.bucket_override, hw_stride, se_stride, int(p.value_norm), float(p.value_norm_eps), int(p.shared_elastic), 0)
+                      p.bucket_override, hw_stride, se_stride, int(p.value_norm), float(p.value_norm_eps), int(p.shared_elastic), int(p.global_alpha),
+                      int(p.units_per_prompt), 0)
 
 
 def _ptr(t):
@@ -211,6 +216,16 @@ def ckv_budget(shape, params, scores, colmass, sens, budgets, offsets, bucket, e
 def ckv_vnorm(shape, params, v, rho, scores, ws, stream=None):
     _check(lib().ckv_vnorm(C.byref(shape), C.byref(params), _ptr(v), _ptr(rho), _ptr(scores), _ptr(ws), ws.numel(),
                            _stream(stream)), "ckv_vnorm")
+
+
+def ckv_prompt_mass(shape, params, colmass, pmass, stream=None):
+    _check(lib().ckv_prompt_mass(C.byref(shape), C.byref(params), _ptr(colmass), _ptr(pmass), _stream(stream)),
+           "ckv_prompt_mass")
+
+
+def ckv_global_scores(shape, params, head_w, pmass, units_total, scores, colmass, stream=None):
+    _check(lib().ckv_global_scores(C.byref(shape), C.byref(params), _ptr(head_w), _ptr(pmass), int(units_total),
+                                   _ptr(scores), _ptr(colmass), _stream(stream)), "ckv_global_scores")
 
 
 def ckv_unit_max(shape, params, scores, stream=None):

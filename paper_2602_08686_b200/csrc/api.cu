@@ -36,6 +36,7 @@ WsLayout ws_layout(const ckv_shape& s, const ckv_params& p) {
     w.cnt_part = o, o = align_up(o + b.cnt_bytes);
     w.bud_done = o, o = align_up(o + b.done_bytes);
   }
+  w.pmass = o, o = align_up(o + (p.global_alpha ? Nu / (size_t)p.units_per_prompt * L * sizeof(float) : 0));
   w.vn_part = o, o = align_up(o + Nu * Hkv * ((L + kVnormRows - 1) / kVnormRows) * sizeof(float));
   w.vn_rho = o, o = align_up(o + (p.value_norm ? Nu * Hkv * L * sizeof(float) : 0));
   if (s.dtype == CKV_BF16) {
@@ -78,6 +79,9 @@ static ckv_status check_params(const ckv_shape* s, const ckv_params* p) {
   if (p->head_w_stride_unit < 0 || p->sens_stride_unit < 0) return CKV_ERR_INVALID_ARG;
   if (p->value_norm != 0 && p->value_norm != 1) return CKV_ERR_INVALID_ARG;
   if (p->shared_elastic != 0 && p->shared_elastic != 1) return CKV_ERR_INVALID_ARG;
+  if (p->global_alpha != 0 && p->global_alpha != 1) return CKV_ERR_INVALID_ARG;
+  if (p->units_per_prompt < 0) return CKV_ERR_INVALID_ARG;
+  if (p->global_alpha && (p->units_per_prompt < 1 || s->n_units % p->units_per_prompt)) return CKV_ERR_INVALID_ARG;
   if (!(p->value_norm_eps >= 0.f) || !(p->value_norm_eps < 3.0e38f)) return CKV_ERR_INVALID_ARG;
   if (p->budget_per_head < s->seq_len) {
     if (p->budget_per_head < s->window) return CKV_ERR_INVALID_ARG;
@@ -192,6 +196,25 @@ ckv_status ckv_vnorm(const ckv_shape* shape, const ckv_params* params, const voi
   return CKV_OK;
 }
 
+ckv_status ckv_prompt_mass(const ckv_shape* shape, const ckv_params* params, const float* colmass, float* pmass,
+                           void* stream) {
+  CKV_TRY(check_shape(shape));
+  CKV_TRY(check_params(shape, params));
+  if (!params->global_alpha || !all_aligned4({colmass, pmass})) return CKV_ERR_INVALID_ARG;
+  CKV_CUDA(launch_prompt_mass(*shape, *params, colmass, pmass, (cudaStream_t)stream));
+  return CKV_OK;
+}
+
+ckv_status ckv_global_scores(const ckv_shape* shape, const ckv_params* params, const float* head_w,
+                             const float* pmass, int32_t units_total, float* scores, float* colmass, void* stream) {
+  CKV_TRY(check_shape(shape));
+  CKV_TRY(check_params(shape, params));
+  if (!params->global_alpha || units_total < params->units_per_prompt) return CKV_ERR_INVALID_ARG;
+  if (!all_aligned4({head_w, pmass, scores, colmass})) return CKV_ERR_INVALID_ARG;
+  CKV_CUDA(launch_global_scores(*shape, *params, units_total, head_w, pmass, scores, colmass, (cudaStream_t)stream));
+  return CKV_OK;
+}
+
 ckv_status ckv_unit_max(const ckv_shape* shape, const ckv_params* params, float* scores, void* stream) {
   CKV_TRY(check_shape(shape));
   CKV_TRY(check_params(shape, params));
@@ -239,6 +262,13 @@ ckv_status ckv_compress(const ckv_shape* shape, const ckv_params* params, const 
   int32_t* bucket = bucket_or_null ? bucket_or_null : reinterpret_cast<int32_t*>(base + w.bucket);
   float* entropy = entropy_or_null ? entropy_or_null : reinterpret_cast<float*>(base + w.entropy);
   CKV_TRY(score_impl(*shape, *params, q_win, k, head_w, scores, colmass, base, st));
+  if (params->global_alpha) {   // Alg. 1 (A): one alpha per prompt, all of whose units are in this call
+    float* pmass = reinterpret_cast<float*>(base + w.pmass);
+    CKV_CUDA(launch_prompt_mass(*shape, *params, colmass, pmass, st));
+    CKV_CUDA(launch_global_scores(*shape, *params, params->units_per_prompt, head_w, pmass, scores, colmass, st));
+    // the pooling kernel left entropy partials of the per-unit mass: redo them for the prompt's
+    CKV_CUDA(launch_entropy_partials(*shape, colmass, base + w.ent_part, base + w.bud_done, st));
+  }
   if (params->value_norm) {   // Eq. 4: u = alpha * rho, before the thresholds see the scores
     float* rho = reinterpret_cast<float*>(base + w.vn_rho);
     float* part = reinterpret_cast<float*>(base + w.vn_part);

@@ -34,6 +34,7 @@ struct WsLayout {
   size_t ent_part; // double [Nu, nblk]        entropy partials of the budget stage (nblk = ceil(L / kEntSpan))
   size_t cnt_part; // int32 [Nu, Hkv, S]       candidate counts per slice
   size_t bud_done; // int32 [Nu]               CTAs of the unit that have finished counting
+  size_t pmass;    // float [Nu / units_per_prompt, L] window mass summed over a prompt's units (only with global_alpha)
   size_t vn_part;  // float [Nu, Hkv, ceil(L / kVnormRows)] block sums of the value-row norms
   size_t vn_rho;   // float [Nu, Hkv, L]       value-norm ratios of the fused call (only with value_norm)
   size_t total;
@@ -95,6 +96,11 @@ cudaError_t launch_budget(const ckv_shape& s, const ckv_params& p, const float* 
 cudaError_t launch_vnorm_rows(const ckv_shape& s, const void* v, float* rho, float* part, cudaStream_t st);
 cudaError_t launch_vnorm_finish(const ckv_shape& s, float eps, float* rho, const float* part, float* scores,
                                 cudaStream_t st);
+// Prompt-global alpha (Alg. 1 (A)): per-prompt sums of the units' column mass, then scores from them.
+cudaError_t launch_prompt_mass(const ckv_shape& s, const ckv_params& p, const float* colmass, float* pmass,
+                               cudaStream_t st);
+cudaError_t launch_global_scores(const ckv_shape& s, const ckv_params& p, int units_total, const float* head_w,
+                                 const float* pmass, float* scores, float* colmass, cudaStream_t st);
 // Eq. 6 over all heads of a unit (the shared elastic selection): scores[u,g,:] <- max_g' scores[u,g',:].
 cudaError_t launch_unit_max(const ckv_shape& s, float* scores, cudaStream_t st);
 cudaError_t launch_select(const ckv_shape& s, const ckv_params& p, const float* scores, const int32_t* budgets,

@@ -44,12 +44,12 @@ def llama_shape(L=32768, W=32, Nu=2, H=32, Hkv=8, d=128, dtype=B.BF16):
 def default_params(**kw):
     base = dict(pool_kind=B.POOL_MAX, pool_size=7, budget_per_head=512, floor_per_head=1, n_buckets=16,
                 bucket_override=-1, head_w_stride_unit=32, sens_stride_unit=0, value_norm=0, value_norm_eps=1e-6,
-                shared_elastic=0, reserved_=0)
+                shared_elastic=0, global_alpha=0, units_per_prompt=1, reserved_=0)
     base.update(kw)
     return B.ckv_params(*[base[k] for k in ("pool_kind", "pool_size", "budget_per_head", "floor_per_head",
                                             "n_buckets", "bucket_override", "head_w_stride_unit",
                                             "sens_stride_unit", "value_norm", "value_norm_eps", "shared_elastic",
-                                            "reserved_")])
+                                            "global_alpha", "units_per_prompt", "reserved_")])
 
 
 def test_argument_errors_are_found_on_the_host():
@@ -73,6 +73,9 @@ def test_argument_errors_are_found_on_the_host():
     assert score(s, default_params(bucket_override=16)) == B.ERR_INVALID_ARG
     assert score(s, default_params(value_norm=2)) == B.ERR_INVALID_ARG
     assert score(s, default_params(shared_elastic=3)) == B.ERR_INVALID_ARG
+    assert score(s, default_params(global_alpha=1, units_per_prompt=3)) == B.ERR_INVALID_ARG   # 2 units
+    assert score(s, default_params(global_alpha=1, units_per_prompt=0)) == B.ERR_INVALID_ARG
+    assert B.ckv_workspace_bytes(s, default_params(global_alpha=1, units_per_prompt=2)) > B.ckv_workspace_bytes(s, p)
     assert score(s, default_params(value_norm_eps=-1.0)) == B.ERR_INVALID_ARG
     assert score(s, default_params(value_norm_eps=float("nan"))) == B.ERR_INVALID_ARG
     assert lib.ckv_vnorm(C.byref(s), C.byref(p), None, fake, None, fake, big, None) == B.ERR_INVALID_ARG
@@ -138,7 +141,7 @@ def test_shard_units_partitions():
 _GLOO_WORKER = r"""
 import os, sys, torch, torch.distributed as dist
 sys.path.insert(0, sys.argv[1])
-from paper_2602_08686_b200.sharding import shard_units, max_over_ranks
+from paper_2602_08686_b200.sharding import shard_units, max_over_ranks, allreduce_prompt_mass
 dist.init_process_group("gloo", init_method="tcp://127.0.0.1:" + sys.argv[2], rank=int(sys.argv[3]), world_size=2)
 rank = dist.get_rank()
 mine = shard_units(33, rank, 2)
@@ -149,6 +152,14 @@ elapsed = max_over_ranks(1.0 + rank)
 assert elapsed == 2.0, elapsed
 total = torch.tensor([float(len(mine))]); dist.all_reduce(total)
 assert total.item() == 33.0
+# prompt-global mode: 3 prompts x 8 layers, each rank holds 4 layers of every prompt; the ranks' partial
+# window masses add up to the sum over all layers (what one process holding all units computes)
+g = torch.Generator().manual_seed(7)
+mass = torch.rand(3, 8, 50, generator=g)                     # [prompt, layer, L], the same on both ranks
+mine_layers = mass[:, 4 * rank: 4 * rank + 4]
+pm = mine_layers.sum(1)                                      # stands in for ckv_prompt_mass on the local units
+allreduce_prompt_mass(pm)
+assert torch.allclose(pm, mass.sum(1), rtol=1e-6), (pm - mass.sum(1)).abs().max()
 dist.barrier(); dist.destroy_process_group()
 print("rank", rank, "ok")
 """
