@@ -43,7 +43,7 @@ def needle_census(cfg, b, idx, bud, off):
     return planted, kept, lost
 
 
-def run_full(B, cfg, units, sample):
+def run_full(B, cfg, units, sample, census=True):
     """One fused call over `units`; oracle comparison on the positions `sample` of that list."""
     b = gen.make_batch(cfg, "cuda", units)
     Nu = len(units)
@@ -83,7 +83,7 @@ def run_full(B, cfg, units, sample):
     # a head share that row its attention is split, so a few fall short of the cut at this scale (the oracle pins
     # the strict form on small cases).  Under heavy-tailed key scales or average pooling other keys pass the
     # needles by design of the workload; there the oracle comparison above is the check.
-    if not cfg.heavy_tail and cfg.pool_kind == 1:
+    if census and not cfg.heavy_tail and cfg.pool_kind == 1:
         planted, kept, lost = needle_census(cfg, b, idx, bud, off)
         assert kept >= 0.99 * planted, (kept, planted, lost[:8])
     del b, out
@@ -114,3 +114,22 @@ def test_config5_sweep(B, L, budget):
     """Qwen2.5-7B shape (GQA 7, W 64, avg pool 5, floor 8, low-reliability heads), batch 4 x 28 layers in one call."""
     cfg = gen.shrink(gen.CONFIGS["c5"], seq_len=L, budget_per_head=budget)
     run_full(B, cfg, list(range(cfg.n_units)), [3, 100] if L <= 16384 else [57])
+
+
+# ------------------------------------------------------------------------------------------ the library's limits
+def test_longest_sequence(B):
+    """seq_len = 2^20 (the largest the library accepts): 8192 key tiles per chunk, the 8-bit-digit selection
+    (prefixes above 262144), 64-bit offsets.  One unit, one KV head, W = 64."""
+    cfg = gen.shrink(gen.CONFIGS["c5"], n_layers=1, batch=1, n_q_heads=2, n_kv_heads=1, seq_len=1 << 20, window=64,
+                     budget_per_head=4096, n_needles=8)
+    run_full(B, cfg, [0], [0])
+
+
+def test_most_kv_heads_and_many_units(B):
+    """64 KV heads (the limit) with one query head each, and a call of 4096 short units."""
+    cfg = gen.shrink(gen.CONFIGS["c2"], n_layers=2, n_q_heads=64, n_kv_heads=64, seq_len=1000, budget_per_head=64,
+                     n_needles=2)
+    run_full(B, cfg, [0, 1], [0, 1], census=False)     # tiny budgets: the oracle comparison is the check
+    cfg = gen.shrink(gen.CONFIGS["c2"], n_layers=4096, n_q_heads=4, n_kv_heads=2, seq_len=160, budget_per_head=48,
+                     n_needles=1)
+    run_full(B, cfg, list(range(4096)), [0, 4095], census=False)
