@@ -321,6 +321,13 @@ def main():
         del staging
 
     # ---- the oracle on the host cores, bounded sample (rank 0, single GPU only) ----------------------
+    # ---- quality of the selection on this synthetic workload (Prop. 4.1's discarded mass; not timed) ----
+    step()
+    kept = torch.empty(n_units, cfg.n_q_heads, cfg.window, device=dev)
+    B.ckv_kept_mass(shape, params, batch["q"], k_out, indices, budgets, offsets, kept, ws)
+    m = (1.0 - kept.double()).clamp_min(0.0)
+    quality = {"mean_discarded_mass": float(m.mean()), "eps_tail": float((m ** 2).mean(-1).sqrt().mean()),
+               "what": "attention mass of the window rows outside the retained set (Prop. 4.1), rank 0's units"}
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         # a first unit gives the oracle's pace; then as many units as fit in about 15 s of wall time
@@ -341,7 +348,8 @@ def main():
                 "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if cfg.dtype == "bf16" else "f32",
                 "data": "synthetic", "config": dict(config_dict(cfg, n_units, world), **({"value_norm": True} if args.value_norm else {})),
                 "clocks": clocks, "e2e": e2e,
-                "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu_baseline}
+                "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu_baseline,
+                "quality": quality}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

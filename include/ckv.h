@@ -139,6 +139,20 @@ ckv_status ckv_vnorm(const ckv_shape* shape, const ckv_params* params, const voi
                      float* scores_or_null, void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * Diagnostic of Prop. 4.1 on the observation-window rows (they stand in for decode queries): the attention mass
+ * that survives the selection,
+ *   kept[u,h,i] = sum over the retained positions t of KV head h/G that row i can see of A^h[n+i, t],
+ * so that m = 1 - kept is the discarded mass, |p - p~|_1 = 2 m for the renormalised restriction p~, and
+ * eps_tail = sqrt(mean_i m^2) enters the Frobenius bound of the proposition.  Computed from the gathered keys k_out
+ * (so it also checks what ckv_gather wrote) and the softmax normalisers that the last ckv_score / ckv_compress
+ * call on this work space left in it; indices, budgets, offsets, k_out as produced by that pass.
+ * kept [Nu,H,W] fp32.  Not part of the retention pass itself.
+ */
+ckv_status ckv_kept_mass(const ckv_shape* shape, const ckv_params* params, const void* q_win, const void* k_out,
+                         const int32_t* indices, const int32_t* budgets, const int32_t* offsets, float* kept, void* ws,
+                         size_t ws_bytes, void* stream);
+
+/*
  * Prompt-global window mass (Alg. 1 (A): A-bar = mean over layers and heads; alpha = (T/W) sum_{j in Omega} A-bar[j,:]),
  * for params->global_alpha.  After ckv_score:
  *   ckv_prompt_mass    pmass[s,t] = sum over the prompt's units in this call of colmass[u,t]; pmass [Nu/N, L] fp32.

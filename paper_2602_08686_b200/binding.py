@@ -64,6 +64,7 @@ def lib() -> C.CDLL:
         L.ckv_select.argtypes = [shp, prm, fp, i32p, i32p, i32p, vp, sz, vp]
         L.ckv_vnorm.argtypes = [shp, prm, vp, fp, fp, vp, sz, vp]
         L.ckv_unit_max.argtypes = [shp, prm, fp, vp]
+        L.ckv_kept_mass.argtypes = [shp, prm, vp, vp, i32p, i32p, i32p, fp, vp, sz, vp]
         L.ckv_prompt_mass.argtypes = [shp, prm, fp, fp, vp]
         L.ckv_global_scores.argtypes = [shp, prm, fp, fp, C.c_int32, fp, fp, vp]
         L.ckv_gather.argtypes = [shp, prm, vp, vp, i32p, i32p, vp, vp, vp]
@@ -78,7 +79,7 @@ def lib() -> C.CDLL:
         L.ckv_status_string.restype = C.c_char_p
         L.ckv_status_string.argtypes = [C.c_int]
         L.ckv_allocate_rows_host.argtypes = [C.c_int, C.c_int64, C.c_int64, C.c_int64, vp, vp]
-        for name in ("ckv_score", "ckv_score_noalloc", "ckv_budget", "ckv_select", "ckv_vnorm", "ckv_unit_max", "ckv_prompt_mass", "ckv_global_scores", "ckv_gather", "ckv_compress", "ckv_compress_host",
+        for name in ("ckv_score", "ckv_score_noalloc", "ckv_budget", "ckv_select", "ckv_vnorm", "ckv_unit_max", "ckv_kept_mass", "ckv_prompt_mass", "ckv_global_scores", "ckv_gather", "ckv_compress", "ckv_compress_host",
                      "ckv_device_status", "ckv_version", "ckv_allocate_rows_host"):
             getattr(L, name).restype = C.c_int
         _lib = L
@@ -226,6 +227,11 @@ def ckv_prompt_mass(shape, params, colmass, pmass, stream=None):
 def ckv_global_scores(shape, params, head_w, pmass, units_total, scores, colmass, stream=None):
     _check(lib().ckv_global_scores(C.byref(shape), C.byref(params), _ptr(head_w), _ptr(pmass), int(units_total),
                                    _ptr(scores), _ptr(colmass), _stream(stream)), "ckv_global_scores")
+
+
+def ckv_kept_mass(shape, params, q_win, k_out, indices, budgets, offsets, kept, ws, stream=None):
+    _check(lib().ckv_kept_mass(C.byref(shape), C.byref(params), _ptr(q_win), _ptr(k_out), _ptr(indices), _ptr(budgets),
+                               _ptr(offsets), _ptr(kept), _ptr(ws), ws.numel(), _stream(stream)), "ckv_kept_mass")
 
 
 def ckv_unit_max(shape, params, scores, stream=None):

@@ -129,6 +129,7 @@ static ckv_status score_impl(const ckv_shape& s, const ckv_params& p, const void
     // grouped output where it applies: both arrays fit the per-head region (at least two heads per group)
     TcGrouped grp{csum, csum + (int64_t)s.n_units * s.n_kv_heads * s.seq_len, head_w, p.head_w_stride_unit};
     const bool grouped = score_tc_groupable(s, p) && g_group_fuse.load(std::memory_order_relaxed) != 0;
+    CKV_CUDA(cudaMemsetAsync(ws + w.status + kPathMarkerWord * sizeof(int), 2, sizeof(int), st));   // who wrote the row statistics
     if (ev0) CKV_CUDA(cudaEventRecord(ev0, st));
     CKV_CUDA(launch_score_tc(s, q, k, csum, grouped ? &grp : nullptr, ws + w.tc_part, ws + w.tc_stat,
                              reinterpret_cast<int*>(ws + w.tc_flags), reinterpret_cast<int*>(ws + w.status), st));
@@ -139,6 +140,7 @@ static ckv_status score_impl(const ckv_shape& s, const ckv_params& p, const void
       return CKV_OK;
     }
   } else {
+    CKV_CUDA(cudaMemsetAsync(ws + w.status + kPathMarkerWord * sizeof(int), 1, sizeof(int), st));
     CKV_CUDA(launch_score_plain(s, q, k, csum, reinterpret_cast<float2*>(ws + w.part),
                                 reinterpret_cast<float2*>(ws + w.stat), w.nblk, st));
   }
@@ -193,6 +195,21 @@ ckv_status ckv_vnorm(const ckv_shape* shape, const ckv_params* params, const voi
   float* part = reinterpret_cast<float*>((char*)ws + w.vn_part);
   CKV_CUDA(launch_vnorm_rows(*shape, v, rho, part, (cudaStream_t)stream));
   CKV_CUDA(launch_vnorm_finish(*shape, params->value_norm_eps, rho, part, scores_or_null, (cudaStream_t)stream));
+  return CKV_OK;
+}
+
+ckv_status ckv_kept_mass(const ckv_shape* shape, const ckv_params* params, const void* q_win, const void* k_out,
+                         const int32_t* indices, const int32_t* budgets, const int32_t* offsets, float* kept, void* ws,
+                         size_t ws_bytes, void* stream) {
+  CKV_TRY(check_shape(shape));
+  CKV_TRY(check_params(shape, params));
+  if (!all_aligned16({q_win, k_out}) || !all_aligned4({indices, budgets, offsets, kept})) return CKV_ERR_INVALID_ARG;
+  CKV_TRY(check_ws(shape, params, ws, ws_bytes));
+  const WsLayout w = ws_layout(*shape, *params);
+  char* base = (char*)ws;
+  CKV_CUDA(launch_kept_mass(*shape, *params, q_win, k_out, indices, budgets, offsets, base + w.stat, base + w.tc_stat,
+                            reinterpret_cast<const int*>(base + w.status) + kPathMarkerWord, kept,
+                            (cudaStream_t)stream));
   return CKV_OK;
 }
 

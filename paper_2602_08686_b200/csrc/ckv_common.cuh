@@ -101,6 +101,13 @@ cudaError_t launch_prompt_mass(const ckv_shape& s, const ckv_params& p, const fl
                                cudaStream_t st);
 cudaError_t launch_global_scores(const ckv_shape& s, const ckv_params& p, int units_total, const float* head_w,
                                  const float* pmass, float* scores, float* colmass, cudaStream_t st);
+// Kept attention mass of the window rows on the retained set (Prop. 4.1's 1 - m), from the gathered keys and the
+// row statistics in the work space; marker tells which scan wrote them (low byte 2: the tensor-core kernel).
+constexpr int kPathMarkerWord = 48;   // index into the work space's 64 status words
+cudaError_t launch_kept_mass(const ckv_shape& s, const ckv_params& p, const void* q, const void* k_out,
+                             const int32_t* indices, const int32_t* budgets, const int32_t* offsets,
+                             const void* stat_plain, const void* stat_tc, const int* marker, float* kept,
+                             cudaStream_t st);
 // Eq. 6 over all heads of a unit (the shared elastic selection): scores[u,g,:] <- max_g' scores[u,g',:].
 cudaError_t launch_unit_max(const ckv_shape& s, float* scores, cudaStream_t st);
 cudaError_t launch_select(const ckv_shape& s, const ckv_params& p, const float* scores, const int32_t* budgets,
