@@ -23,6 +23,7 @@ WsLayout ws_layout(const ckv_shape& s, const ckv_params& p) {
   w.nblk = (int)((L + kPlainKeysPerBlock - 1) / kPlainKeysPerBlock);
   size_t o = 0;
   w.status = o, o += 256;
+  if (s.dtype == CKV_BF16) w.tc_flags = o, o = align_up(o + tc_layout(s).flag_bytes);   // behind the status words: one memset clears both
   w.csum = o, o = align_up(o + Nu * H * L * sizeof(float));
   w.part = o, o = align_up(o + Nu * H * W * (size_t)w.nblk * sizeof(float2));
   w.stat = o, o = align_up(o + Nu * H * W * sizeof(float2));
@@ -43,7 +44,6 @@ WsLayout ws_layout(const ckv_shape& s, const ckv_params& p) {
     const TcLayout t = tc_layout(s);
     w.tc_part = o, o = align_up(o + t.part_bytes);
     w.tc_stat = o, o = align_up(o + t.stat_bytes);
-    w.tc_flags = o, o = align_up(o + t.flag_bytes);
   }
   w.total = o;
   return w;
@@ -119,32 +119,34 @@ static bool all_aligned4(std::initializer_list<const void*> ps) {
 static ckv_status score_impl(const ckv_shape& s, const ckv_params& p, const void* q, const void* k,
                              const float* head_w, float* scores, float* colmass, char* ws, cudaStream_t st) {
   const WsLayout w = ws_layout(s, p);
-  CKV_CUDA(cudaMemsetAsync(ws + w.status, 0, 256, st));
-  float* csum = reinterpret_cast<float*>(ws + w.csum);
   const int path = g_score_path.load(std::memory_order_relaxed);
   const bool tc_ok = score_tc_supported(s) && s.seq_len >= 128;
   if (path == 2 && !tc_ok) return CKV_ERR_UNSUPPORTED;
+  const bool use_tc = tc_ok && path != 1;
+  // the status words and, behind them, the tensor-core scan's counters and run queues
+  CKV_CUDA(cudaMemsetAsync(ws + w.status, 0, 256 + (use_tc ? tc_layout(s).flag_bytes : 0), st));
+  float* csum = reinterpret_cast<float*>(ws + w.csum);
   const cudaEvent_t ev0 = g_scan_start.load(), ev1 = g_scan_stop.load();
-  if (tc_ok && path != 1) {
+  int* marker = reinterpret_cast<int*>(ws + w.status) + kPathMarkerWord;   // who wrote the row statistics
+  if (use_tc) {
     // grouped output where it applies: both arrays fit the per-head region (at least two heads per group)
     TcGrouped grp{csum, csum + (int64_t)s.n_units * s.n_kv_heads * s.seq_len, head_w, p.head_w_stride_unit};
     const bool grouped = score_tc_groupable(s, p) && g_group_fuse.load(std::memory_order_relaxed) != 0;
-    CKV_CUDA(cudaMemsetAsync(ws + w.status + kPathMarkerWord * sizeof(int), 2, sizeof(int), st));   // who wrote the row statistics
     if (ev0) CKV_CUDA(cudaEventRecord(ev0, st));
     CKV_CUDA(launch_score_tc(s, q, k, csum, grouped ? &grp : nullptr, ws + w.tc_part, ws + w.tc_stat,
                              reinterpret_cast<int*>(ws + w.tc_flags), reinterpret_cast<int*>(ws + w.status), st));
     if (ev1) CKV_CUDA(cudaEventRecord(ev1, st));
     if (grouped) {
       CKV_CUDA(launch_epilogue_grouped(s, p, grp.zgrp, grp.mgrp, scores, colmass, ws + w.ent_part, ws + w.bud_done,
-                                       st));
+                                       marker, 2, st));
       return CKV_OK;
     }
   } else {
-    CKV_CUDA(cudaMemsetAsync(ws + w.status + kPathMarkerWord * sizeof(int), 1, sizeof(int), st));
     CKV_CUDA(launch_score_plain(s, q, k, csum, reinterpret_cast<float2*>(ws + w.part),
                                 reinterpret_cast<float2*>(ws + w.stat), w.nblk, st));
   }
-  CKV_CUDA(launch_epilogue(s, p, csum, head_w, scores, colmass, ws + w.ent_part, ws + w.bud_done, st));
+  CKV_CUDA(launch_epilogue(s, p, csum, head_w, scores, colmass, ws + w.ent_part, ws + w.bud_done, marker,
+                           use_tc ? 2 : 1, st));
   return CKV_OK;
 }
 

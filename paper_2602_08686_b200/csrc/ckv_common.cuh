@@ -68,6 +68,7 @@ struct TcGrouped {
   int64_t hw_stride;
 };
 bool score_tc_groupable(const ckv_shape& s, const ckv_params& p);
+// flags must be zero at launch (tc_layout's flag_bytes).
 cudaError_t launch_score_tc(const ckv_shape& s, const void* q, const void* k, float* csum, const TcGrouped* grp,
                             void* part, void* stat, int* flags, int* status, cudaStream_t st);
 
@@ -78,13 +79,16 @@ void count_launch(int n = 1);
 // Launchers; each returns cudaGetLastError() after queuing its kernels.
 cudaError_t launch_score_plain(const ckv_shape& s, const void* q, const void* k, float* csum, float2* part,
                                float2* stat, int nblk, cudaStream_t st);
-// The epilogue also leaves the budget stage's entropy partials (one per kEntSpan positions) and clears its
+// The epilogue also writes marker_value to *marker (which scan produced the row statistics in the work space),
+// leaves the budget stage's entropy partials (one per kEntSpan positions) and clears its
 // arrival counters; launch_entropy_partials does the same from a column mass the caller supplies.
 cudaError_t launch_epilogue(const ckv_shape& s, const ckv_params& p, const float* csum, const float* head_w,
-                            float* scores, float* colmass, void* ent_part, void* done, cudaStream_t st);
+                            float* scores, float* colmass, void* ent_part, void* done, int* marker, int marker_value,
+                            cudaStream_t st);
 // The same from the scan's grouped output: pooling of zgrp inside the prefix, column mass from mgrp.
 cudaError_t launch_epilogue_grouped(const ckv_shape& s, const ckv_params& p, const float* zgrp, const float* mgrp,
-                                    float* scores, float* colmass, void* ent_part, void* done, cudaStream_t st);
+                                    float* scores, float* colmass, void* ent_part, void* done, int* marker,
+                                    int marker_value, cudaStream_t st);
 cudaError_t launch_entropy_partials(const ckv_shape& s, const float* colmass, void* ent_part, void* done,
                                     cudaStream_t st);
 // Expects the entropy partials and cleared counters of one of the two launchers above.

@@ -64,7 +64,8 @@ __global__ void __launch_bounds__(kThreads) pool_weight_max_mass(ckv_shape s, ck
                                                                  float* __restrict__ scores,
                                                                  float* __restrict__ colmass,
                                                                  double* __restrict__ ent_part,
-                                                                 int* __restrict__ done) {
+                                                                 int* __restrict__ done, int* __restrict__ marker,
+                                                                 int marker_value) {
   constexpr int kHalo = (R + 3) / 4 * 4;           // halo rounded up so that every thread's window is 16-byte aligned
   constexpr int kWidth = kSpan + 2 * kHalo;        // staged positions t0 - kHalo .. t0 + kSpan + kHalo - 1
   constexpr int kWin = kPerThread + 2 * kHalo;     // values a thread reads: c_h[tb - kHalo .. tb + 3 + kHalo]
@@ -172,22 +173,23 @@ __global__ void __launch_bounds__(kThreads) pool_weight_max_mass(ckv_shape s, ck
   if (threadIdx.x == 0) {
     ent_part[(int64_t)u * gridDim.x + blockIdx.x] = tot;
     if (blockIdx.x == 0) done[u] = 0;
+    if (blockIdx.x == 0 && u == 0) *marker = marker_value;
   }
 }
 
 template <int R>
 void launch_r(bool avg, dim3 grid, cudaStream_t st, const ckv_shape& s, const ckv_params& p, const float* csum,
-              const float* head_w, float* scores, float* colmass, double* ent, int* done) {
+              const float* head_w, float* scores, float* colmass, double* ent, int* done, int* mk, int mv) {
   if (avg)
-    pool_weight_max_mass<R, true, false><<<grid, kThreads, 0, st>>>(s, p, csum, nullptr, head_w, scores, colmass, ent, done);
+    pool_weight_max_mass<R, true, false><<<grid, kThreads, 0, st>>>(s, p, csum, nullptr, head_w, scores, colmass, ent, done, mk, mv);
   else
-    pool_weight_max_mass<R, false, false><<<grid, kThreads, 0, st>>>(s, p, csum, nullptr, head_w, scores, colmass, ent, done);
+    pool_weight_max_mass<R, false, false><<<grid, kThreads, 0, st>>>(s, p, csum, nullptr, head_w, scores, colmass, ent, done, mk, mv);
 }
 
 template <int R>
 void launch_g(dim3 grid, cudaStream_t st, const ckv_shape& s, const ckv_params& p, const float* zgrp,
-              const float* mgrp, float* scores, float* colmass, double* ent, int* done) {
-  pool_weight_max_mass<R, false, true><<<grid, kThreads, 0, st>>>(s, p, zgrp, mgrp, nullptr, scores, colmass, ent, done);
+              const float* mgrp, float* scores, float* colmass, double* ent, int* done, int* mk, int mv) {
+  pool_weight_max_mass<R, false, true><<<grid, kThreads, 0, st>>>(s, p, zgrp, mgrp, nullptr, scores, colmass, ent, done, mk, mv);
 }
 
 }  // namespace
@@ -201,41 +203,43 @@ cudaError_t launch_entropy_partials(const ckv_shape& s, const float* colmass, vo
 }
 
 cudaError_t launch_epilogue(const ckv_shape& s, const ckv_params& p, const float* csum, const float* head_w,
-                            float* scores, float* colmass, void* ent_part, void* done, cudaStream_t st) {
+                            float* scores, float* colmass, void* ent_part, void* done, int* marker, int marker_value,
+                            cudaStream_t st) {
   double* ent = (double*)ent_part;
   int* dn = (int*)done;
   dim3 grid((s.seq_len + kSpan - 1) / kSpan, s.n_units);
   const int r = (p.pool_kind == CKV_POOL_NONE) ? 0 : p.pool_size / 2;
   const bool avg = p.pool_kind == CKV_POOL_AVG && r > 0;
   switch (r) {
-    case 0: launch_r<0>(false, grid, st, s, p, csum, head_w, scores, colmass, ent, dn); break;
-    case 1: launch_r<1>(avg, grid, st, s, p, csum, head_w, scores, colmass, ent, dn); break;
-    case 2: launch_r<2>(avg, grid, st, s, p, csum, head_w, scores, colmass, ent, dn); break;
-    case 3: launch_r<3>(avg, grid, st, s, p, csum, head_w, scores, colmass, ent, dn); break;
-    case 4: launch_r<4>(avg, grid, st, s, p, csum, head_w, scores, colmass, ent, dn); break;
-    case 5: launch_r<5>(avg, grid, st, s, p, csum, head_w, scores, colmass, ent, dn); break;
-    case 6: launch_r<6>(avg, grid, st, s, p, csum, head_w, scores, colmass, ent, dn); break;
-    default: launch_r<7>(avg, grid, st, s, p, csum, head_w, scores, colmass, ent, dn); break;
+    case 0: launch_r<0>(false, grid, st, s, p, csum, head_w, scores, colmass, ent, dn, marker, marker_value); break;
+    case 1: launch_r<1>(avg, grid, st, s, p, csum, head_w, scores, colmass, ent, dn, marker, marker_value); break;
+    case 2: launch_r<2>(avg, grid, st, s, p, csum, head_w, scores, colmass, ent, dn, marker, marker_value); break;
+    case 3: launch_r<3>(avg, grid, st, s, p, csum, head_w, scores, colmass, ent, dn, marker, marker_value); break;
+    case 4: launch_r<4>(avg, grid, st, s, p, csum, head_w, scores, colmass, ent, dn, marker, marker_value); break;
+    case 5: launch_r<5>(avg, grid, st, s, p, csum, head_w, scores, colmass, ent, dn, marker, marker_value); break;
+    case 6: launch_r<6>(avg, grid, st, s, p, csum, head_w, scores, colmass, ent, dn, marker, marker_value); break;
+    default: launch_r<7>(avg, grid, st, s, p, csum, head_w, scores, colmass, ent, dn, marker, marker_value); break;
   }
   count_launch();
   return cudaGetLastError();
 }
 
 cudaError_t launch_epilogue_grouped(const ckv_shape& s, const ckv_params& p, const float* zgrp, const float* mgrp,
-                                    float* scores, float* colmass, void* ent_part, void* done, cudaStream_t st) {
+                                    float* scores, float* colmass, void* ent_part, void* done, int* marker,
+                                    int marker_value, cudaStream_t st) {
   double* ent = (double*)ent_part;
   int* dn = (int*)done;
   dim3 grid((s.seq_len + kSpan - 1) / kSpan, s.n_units);
   const int r = (p.pool_kind == CKV_POOL_NONE) ? 0 : p.pool_size / 2;
   switch (r) {
-    case 0: launch_g<0>(grid, st, s, p, zgrp, mgrp, scores, colmass, ent, dn); break;
-    case 1: launch_g<1>(grid, st, s, p, zgrp, mgrp, scores, colmass, ent, dn); break;
-    case 2: launch_g<2>(grid, st, s, p, zgrp, mgrp, scores, colmass, ent, dn); break;
-    case 3: launch_g<3>(grid, st, s, p, zgrp, mgrp, scores, colmass, ent, dn); break;
-    case 4: launch_g<4>(grid, st, s, p, zgrp, mgrp, scores, colmass, ent, dn); break;
-    case 5: launch_g<5>(grid, st, s, p, zgrp, mgrp, scores, colmass, ent, dn); break;
-    case 6: launch_g<6>(grid, st, s, p, zgrp, mgrp, scores, colmass, ent, dn); break;
-    default: launch_g<7>(grid, st, s, p, zgrp, mgrp, scores, colmass, ent, dn); break;
+    case 0: launch_g<0>(grid, st, s, p, zgrp, mgrp, scores, colmass, ent, dn, marker, marker_value); break;
+    case 1: launch_g<1>(grid, st, s, p, zgrp, mgrp, scores, colmass, ent, dn, marker, marker_value); break;
+    case 2: launch_g<2>(grid, st, s, p, zgrp, mgrp, scores, colmass, ent, dn, marker, marker_value); break;
+    case 3: launch_g<3>(grid, st, s, p, zgrp, mgrp, scores, colmass, ent, dn, marker, marker_value); break;
+    case 4: launch_g<4>(grid, st, s, p, zgrp, mgrp, scores, colmass, ent, dn, marker, marker_value); break;
+    case 5: launch_g<5>(grid, st, s, p, zgrp, mgrp, scores, colmass, ent, dn, marker, marker_value); break;
+    case 6: launch_g<6>(grid, st, s, p, zgrp, mgrp, scores, colmass, ent, dn, marker, marker_value); break;
+    default: launch_g<7>(grid, st, s, p, zgrp, mgrp, scores, colmass, ent, dn, marker, marker_value); break;
   }
   count_launch();
   return cudaGetLastError();

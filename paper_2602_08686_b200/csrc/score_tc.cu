@@ -993,8 +993,7 @@ cudaError_t launch_score_tc(const ckv_shape& s, const void* q, const void* k, fl
     const cuuint32_t box[5] = {64, kTile, 2, 1, 1};
     if (!make_map5(&km, k, dims, strides, box)) return cudaErrorInvalidValue;
   }
-  cudaError_t e = cudaMemsetAsync(flags, 0, t.flag_bytes, st);
-  if (e != cudaSuccess) return e;
+  cudaError_t e;   // flags: zeroed by the caller
   if (a.W == 16) e = launch_w<16>(qm, km, a, grid, st);
   else if (a.W == 32) e = launch_w<32>(qm, km, a, grid, st);
   else e = launch_w<64>(qm, km, a, grid, st);
