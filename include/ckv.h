@@ -273,7 +273,10 @@ void ckv_set_scan_events(void* start_event, void* stop_event);
  *                    (Eq. 6) and adds their column mass, and the pooling runs on that one row per group;
  *                    the scores are bit-identical to the per-head order of operations for head_w >= 0,
  *                    the column mass may differ in the last bit (heads are added group by group);
- *                    0: always write per-head column sums.
+ *                    0: always write per-head column sums;
+ *   "pdl"            1 (default): the counting, selection and gather kernels are launched with programmatic
+ *                    stream serialisation, so each is scheduled while its predecessor drains and waits on the
+ *                    device for it to complete; 0: ordinary launches.
  * Returns the previous value, or -1 for an unknown name or a value out of range. */
 int ckv_set_tunable(const char* name, int value);
 

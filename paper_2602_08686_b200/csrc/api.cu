@@ -10,6 +10,8 @@ namespace ckv {
 
 static std::atomic<int64_t> g_launches{0};
 static std::atomic<int> g_score_path{0};  // 0 = automatic, 1 = plain kernels, 2 = tensor-core kernel
+static std::atomic<int> g_pdl{1};         // 1: the kernels after the pooling kernel use programmatic dependent launch
+bool pdl_enabled() { return g_pdl.load(std::memory_order_relaxed) != 0; }
 static std::atomic<int> g_group_fuse{1};  // 1: the scan writes per-group maxima and masses where it can
 static std::atomic<cudaEvent_t> g_scan_start{nullptr}, g_scan_stop{nullptr};  // see ckv_set_scan_events
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
@@ -404,6 +406,7 @@ void ckv_set_scan_events(void* start_event, void* stop_event) {
 int ckv_set_tunable(const char* name, int value) {
   if (!name) return -1;
   if (std::string(name) == "group_fuse") return g_group_fuse.exchange(value != 0 ? 1 : 0);
+  if (std::string(name) == "pdl") return g_pdl.exchange(value != 0 ? 1 : 0);
   return set_tc_tunable(name, value);
 }
 

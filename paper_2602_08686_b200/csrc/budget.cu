@@ -95,6 +95,8 @@ __global__ void __launch_bounds__(kThreads) count_allocate(ckv_shape s, ckv_para
   __shared__ int last_s;
   __shared__ long long dem_s[kMaxKvHeads], e_s[kMaxKvHeads];
   __shared__ int raw_s;   // candidates of head 0 (the shared elastic selection gives every head the same scores)
+  pdl_launch_dependents();
+  pdl_wait();   // scores and entropy partials come from the kernel before
   const int u = blockIdx.y, L = s.seq_len, W = s.window, n = L - W, Hkv = s.n_kv_heads;
   const int g = blockIdx.x / S, slice = blockIdx.x - g * S;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -217,11 +219,15 @@ cudaError_t launch_budget(const ckv_shape& s, const ckv_params& p, const float* 
                           int32_t* budgets, int32_t* offsets, int32_t* bucket, float* entropy, void* ent_part,
                           void* cnt_part, void* done, cudaStream_t st) {
   const BudgetLayout b = budget_layout(s);
-  count_allocate<<<dim3(s.n_kv_heads * b.S, s.n_units), kThreads, 0, st>>>(
-      s, p, b.S, b.nblk, scores, sens, (const double*)ent_part, (int*)cnt_part, (int*)done, budgets, offsets, bucket,
-      entropy);
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(s.n_kv_heads * b.S, s.n_units), cfg.blockDim = dim3(kThreads), cfg.stream = st;
+  cudaLaunchAttribute attr = pdl_attribute();
+  cfg.attrs = &attr, cfg.numAttrs = 1;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, count_allocate, s, p, b.S, b.nblk, scores, sens,
+                                           (const double*)ent_part, (int*)cnt_part, (int*)done, budgets, offsets,
+                                           bucket, entropy);
   count_launch();
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace ckv

@@ -76,6 +76,20 @@ WsLayout ws_layout(const ckv_shape& s, const ckv_params& p);
 
 void count_launch(int n = 1);
 
+// Programmatic dependent launch between the small kernels that follow the scan: a kernel launched with
+// pdl_attribute() may be scheduled while its predecessor in the stream drains, and must call pdl_wait() before it
+// touches anything the predecessor wrote (or reads what it will overwrite); a predecessor lets it start early with
+// pdl_launch_dependents().  Both are no-ops in a kernel launched the ordinary way.
+bool pdl_enabled();
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+inline cudaLaunchAttribute pdl_attribute() {
+  cudaLaunchAttribute a{};
+  a.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  a.val.programmaticStreamSerializationAllowed = pdl_enabled() ? 1 : 0;
+  return a;
+}
+
 // Launchers; each returns cudaGetLastError() after queuing its kernels.
 cudaError_t launch_score_plain(const ckv_shape& s, const void* q, const void* k, float* csum, float2* part,
                                float2* stat, int nblk, cudaStream_t st);

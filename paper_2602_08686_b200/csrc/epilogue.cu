@@ -66,6 +66,7 @@ __global__ void __launch_bounds__(kThreads) pool_weight_max_mass(ckv_shape s, ck
                                                                  double* __restrict__ ent_part,
                                                                  int* __restrict__ done, int* __restrict__ marker,
                                                                  int marker_value) {
+  pdl_launch_dependents();   // the counting kernel may be scheduled while this grid drains
   constexpr int kHalo = (R + 3) / 4 * 4;           // halo rounded up so that every thread's window is 16-byte aligned
   constexpr int kWidth = kSpan + 2 * kHalo;        // staged positions t0 - kHalo .. t0 + kSpan + kHalo - 1
   constexpr int kWin = kPerThread + 2 * kHalo;     // values a thread reads: c_h[tb - kHalo .. tb + 3 + kHalo]

@@ -11,6 +11,7 @@ __global__ void __launch_bounds__(256) gather_kernel(ckv_shape s, int rows_per_h
                                                      const int32_t* __restrict__ indices,
                                                      const int32_t* __restrict__ offsets, uint4* __restrict__ k_out,
                                                      uint4* __restrict__ v_out) {
+  pdl_wait();   // indices and offsets come from the kernels before
   const int Hkv = s.n_kv_heads;
   const int64_t rows_per_unit = (int64_t)Hkv * rows_per_head;
   const int64_t total = (int64_t)s.n_units * rows_per_unit * vec_per_row;
@@ -50,10 +51,14 @@ cudaError_t launch_gather(const ckv_shape& s, const ckv_params& p, const void* k
   int64_t blocks = (total + 255) / 256;
   if (blocks > 148 * 16) blocks = 148 * 16;
   if (blocks < 1) blocks = 1;
-  gather_kernel<<<(int)blocks, 256, 0, st>>>(s, rows_per_head, vec_per_row, (const uint4*)k, (const uint4*)v, indices,
-                                             offsets, (uint4*)k_out, (uint4*)v_out);
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)blocks), cfg.blockDim = dim3(256), cfg.stream = st;
+  cudaLaunchAttribute attr = pdl_attribute();
+  cfg.attrs = &attr, cfg.numAttrs = 1;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, gather_kernel, s, rows_per_head, vec_per_row, (const uint4*)k,
+                                           (const uint4*)v, indices, offsets, (uint4*)k_out, (uint4*)v_out);
   count_launch();
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace ckv

@@ -66,6 +66,8 @@ __global__ void __launch_bounds__(kThreads) select_sliced_kernel(ckv_shape s, in
   __shared__ uint2 wcnt[2][kCluster][kWarps];
   __shared__ uint32_t wtot[kWarps];
   __shared__ uint32_t ctot[kCluster];
+  pdl_launch_dependents();
+  pdl_wait();   // budgets, offsets and scores come from the kernels before
   const int Hkv = s.n_kv_heads, W = s.window, n = s.seq_len - W;
   const int head = blockIdx.x / kCluster, rank = blockIdx.x % kCluster;
   const int u = head / Hkv, g = head % Hkv;
@@ -204,6 +206,8 @@ __global__ void __launch_bounds__(kThreads) select_digit_kernel(ckv_shape s, int
   __shared__ uint32_t sh_prefix;
   __shared__ int sh_want;
   __shared__ int warp_gt[kWarps], warp_eq[kWarps];
+  pdl_launch_dependents();
+  pdl_wait();
   const int Hkv = s.n_kv_heads, W = s.window, n = s.seq_len - W;
   const int u = blockIdx.x / Hkv, g = blockIdx.x % Hkv;
   const int e = budgets[(int64_t)u * Hkv + g] - W;
@@ -342,10 +346,11 @@ cudaError_t launch_sliced(const ckv_shape& s, int n, int64_t unit_rows, const fl
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = kCluster == 1 ? smem : kSlicedMax * sizeof(uint32_t);
   cfg.stream = st;
-  cudaLaunchAttribute attr{};
-  attr.id = cudaLaunchAttributeClusterDimension;
-  attr.val.clusterDim.x = kCluster, attr.val.clusterDim.y = 1, attr.val.clusterDim.z = 1;
-  cfg.attrs = &attr, cfg.numAttrs = 1;
+  cudaLaunchAttribute attr[2] = {};
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = kCluster, attr[0].val.clusterDim.y = 1, attr[0].val.clusterDim.z = 1;
+  attr[1] = pdl_attribute();
+  cfg.attrs = attr, cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, select_sliced_kernel<kCluster>, s, unit_rows, scores, budgets, offsets, indices);
 }
 
@@ -362,8 +367,11 @@ cudaError_t launch_select(const ckv_shape& s, const ckv_params& p, const float* 
   else if (n <= 4 * kSlicedMax) e = launch_sliced<4>(s, n, unit_rows, scores, budgets, offsets, indices, st);
   else if (n <= 8 * kSlicedMax) e = launch_sliced<8>(s, n, unit_rows, scores, budgets, offsets, indices, st);
   else {
-    select_digit_kernel<<<s.n_units * s.n_kv_heads, kThreads, 0, st>>>(s, unit_rows, scores, budgets, offsets, indices);
-    e = cudaGetLastError();
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(s.n_units * s.n_kv_heads), cfg.blockDim = dim3(kThreads), cfg.stream = st;
+    cudaLaunchAttribute attr = pdl_attribute();
+    cfg.attrs = &attr, cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, select_digit_kernel, s, unit_rows, scores, budgets, offsets, indices);
   }
   count_launch();
   return e != cudaSuccess ? e : cudaGetLastError();
