@@ -254,5 +254,23 @@ def kept_mass(prob: Problem, q, k, indices, budgets, offsets) -> np.ndarray:
     return kept
 
 
+def attend(prob: Problem, q_dec, k, v, budgets=None, offsets=None):
+    """(out [Nu,H,n_dec,d], lse [Nu,H,n_dec]) in fp64: attention of decode queries q_dec [Nu,H,n_dec,d] over all
+    L rows of k, v, or -- when budgets and offsets are given -- over the gathered rows k_out, v_out [Nu, rows, d]."""
+    q_dec, k, v = _inp(q_dec, prob), _inp(k, prob), _inp(v, prob)
+    n_dec = q_dec.shape[2]
+    out = np.empty(q_dec.shape, np.float64)
+    lse = np.empty(q_dec.shape[:3], np.float64)
+    compressed = budgets is not None
+    if compressed:
+        budgets = np.ascontiguousarray(budgets, np.int32)
+        offsets = np.ascontiguousarray(offsets, np.int32)
+    s = prob._shape()
+    _check(lib().oracle_attend(C.byref(s), _p(q_dec), C.c_int(n_dec), _p(k), _p(v), C.c_int(int(compressed)),
+                               _p(budgets), _p(offsets), C.c_int64(k.shape[1] if compressed else 0), _p(out), _p(lse)),
+           "attend")
+    return out, lse
+
+
 def num_threads() -> int:
     return int(lib().oracle_num_threads())

@@ -531,6 +531,47 @@ int oracle_compress(const or_shape *s, const or_params *p, const void *q, const 
   return rc;
 }
 
+/* ------------------------------------------------------------------ decode-side check (Prop. 4.1)
+ * Softmax attention of n_dec decode queries per query head over a K/V array.  A decode query comes after the
+ * prompt and sees every row.  compressed == 0: the rows are all L tokens of k, v [Nu,Hkv,L,d].  compressed == 1:
+ * k, v are the gathered k_out, v_out [Nu, unit_rows, d] and head g of unit u owns budgets[u,g] rows from row
+ * offsets[u,g].  out[u,h,j,:] = sum_t p_t v_t with p = softmax(q.k_t / sqrt d);  lse[u,h,j] = ln sum_t exp(q.k_t / sqrt d).
+ * The mass a restriction to a subset S keeps is sum_{t in S} p_t = exp(lse_S - lse_all). */
+int oracle_attend(const or_shape *s, const void *q_dec, int n_dec, const void *k, const void *v, int compressed,
+                  const int32_t *budgets, const int32_t *offsets, int64_t unit_rows, double *out, double *lse) {
+  const int L = s->seq_len, H = s->n_q_heads, Hkv = s->n_kv_heads, G = H / Hkv, d = s->head_dim;
+#pragma omp parallel for collapse(2) schedule(dynamic)
+  for (int u = 0; u < s->n_units; ++u)
+    for (int h = 0; h < H; ++h) {
+      const int g = h / G;
+      const int64_t rows = compressed ? budgets[(int64_t)u * Hkv + g] : L;
+      const int64_t base = compressed ? (int64_t)u * unit_rows + offsets[(int64_t)u * (Hkv + 1) + g]
+                                      : ((int64_t)u * Hkv + g) * (int64_t)L;
+      double *x = (double *)malloc(sizeof(double) * (size_t)(rows > 0 ? rows : 1));
+      for (int j = 0; j < n_dec; ++j) {
+        const int64_t qo = (((int64_t)u * H + h) * n_dec + j) * d;
+        double mx = -INFINITY;
+        for (int64_t t = 0; t < rows; ++t) {
+          double dot = 0.0;
+          for (int c = 0; c < d; ++c) dot += widen(q_dec, s->dtype, qo + c) * widen(k, s->dtype, (base + t) * d + c);
+          x[t] = dot / sqrt((double)d);
+          if (x[t] > mx) mx = x[t];
+        }
+        double z = 0.0;
+        for (int64_t t = 0; t < rows; ++t) z += exp(x[t] - mx);
+        double *o = out + qo;
+        for (int c = 0; c < d; ++c) o[c] = 0.0;
+        for (int64_t t = 0; t < rows; ++t) {
+          const double p = exp(x[t] - mx) / z;
+          for (int c = 0; c < d; ++c) o[c] += p * widen(v, s->dtype, (base + t) * d + c);
+        }
+        lse[((int64_t)u * H + h) * n_dec + j] = mx + log(z);
+      }
+      free(x);
+    }
+  return 0;
+}
+
 /* ------------------------------------------------------------------ diagnostic (Prop. 4.1)
  * kept[u,h,i] = sum_{t in S_g} A[h,i,t]: attention mass of window row i that
  * survives the selection; the discarded mass is m = 1 - kept. */

@@ -595,3 +595,42 @@ def test_global_alpha_pools_alpha_and_shares_the_risk_coordinate():
     bud = oracle.budget(prob, sc, cm, gen.as_numpy(gen.make_sens(gen.CONFIGS["c1"])))
     assert bud["bucket"][0] == bud["bucket"][1] and bud["bucket"][2] == bud["bucket"][3]
     assert bud["entropy"][0] == bud["entropy"][1]
+
+
+# ---------------------------------------------------------------------------- decode-side check (Prop. 4.1)
+@pytest.mark.parametrize("dtype", [oracle.F32, oracle.BF16])
+def test_attend_against_library_softmax_and_the_discarded_mass_identity(dtype):
+    """Full attention of decode queries equals torch's fp64 softmax attention; over the gathered rows it is the
+    renormalised restriction p~ of Prop. 4.1, the kept mass is exp(lse_S - lse_all), |p - p~|_1 = 2 m (Eq. A2),
+    and keeping every row changes nothing."""
+    prob, q, k, v = rand_case(41, Nu=2, H=4, Hkv=2, L=60, W=6, d=16, dtype=dtype)
+    g = torch.Generator().manual_seed(4)
+    qd = torch.randn(2, 4, 3, 16, generator=g)
+    if dtype == oracle.BF16:
+        qd = qd.bfloat16()
+    kk, vv = k.double().repeat_interleave(2, 1), v.double().repeat_interleave(2, 1)       # [Nu,H,L,d]
+    x = torch.einsum("uhjd,uhtd->uhjt", qd.double(), kk) / 4.0
+    p = torch.softmax(x, -1)
+    out, lse = oracle.attend(prob, gen.as_numpy(qd), gen.as_numpy(k), gen.as_numpy(v))
+    np.testing.assert_allclose(out, torch.einsum("uhjt,uhtd->uhjd", p, vv).numpy(), rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(lse, torch.logsumexp(x, -1).numpy(), rtol=1e-12)
+    # a selection by the retention pass, then attention over what it gathered
+    w = np.ones((2, 4), np.float32)
+    sel = oracle.compress(prob, gen.as_numpy(q), gen.as_numpy(k), gen.as_numpy(v), w, np.zeros(prob.n_buckets, np.float32))
+    out_c, lse_c = oracle.attend(prob, gen.as_numpy(qd), sel["k_out"], sel["v_out"], sel["budgets"], sel["offsets"])
+    for u in range(2):
+        for h in range(4):
+            gq = h // 2
+            S = sel["indices"][u, sel["offsets"][u, gq]: sel["offsets"][u, gq + 1]]
+            pS = p[u, h][:, S]                                   # [n_dec, |S|]
+            kept = pS.sum(-1).numpy()
+            np.testing.assert_allclose(np.exp(lse_c[u, h] - lse[u, h]), kept, rtol=1e-11)
+            p_tilde = torch.zeros_like(p[u, h])
+            p_tilde[:, S] = pS / pS.sum(-1, keepdim=True)
+            np.testing.assert_allclose((p[u, h] - p_tilde).abs().sum(-1).numpy(), 2 * (1 - kept), rtol=1e-9, atol=1e-13)
+            np.testing.assert_allclose(out_c[u, h], (p_tilde @ vv[u, h]).numpy(), rtol=1e-10, atol=1e-13)
+    prob.budget_per_head = 60                                    # FullKV: the compressed cache is the cache
+    full = oracle.compress(prob, gen.as_numpy(q), gen.as_numpy(k), gen.as_numpy(v), w, np.zeros(prob.n_buckets, np.float32))
+    out_f, lse_f = oracle.attend(prob, gen.as_numpy(qd), full["k_out"], full["v_out"], full["budgets"], full["offsets"])
+    np.testing.assert_allclose(out_f, out, rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(lse_f, lse, rtol=1e-13)
