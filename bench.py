@@ -328,6 +328,20 @@ def main():
     m = (1.0 - kept.double()).clamp_min(0.0)
     quality = {"mean_discarded_mass": float(m.mean()), "eps_tail": float((m ** 2).mean(-1).sqrt().mean()),
                "what": "attention mass of the window rows outside the retained set (Prop. 4.1), rank 0's units"}
+    n_dec = max(1, min(4, 32 // (cfg.n_q_heads // cfg.n_kv_heads)))
+    gq = torch.Generator(device=dev)
+    gq.manual_seed(4242)
+    q_dec = torch.randn(n_units, cfg.n_q_heads, n_dec, cfg.head_dim, generator=gq, device=dev).to(batch["q"].dtype)
+    o_f = torch.empty(n_units, cfg.n_q_heads, n_dec, cfg.head_dim, device=dev)
+    o_c = torch.empty_like(o_f)
+    l_f = torch.empty(n_units, cfg.n_q_heads, n_dec, device=dev)
+    l_c = torch.empty_like(l_f)
+    B.ckv_attend(shape, params, q_dec, batch["k"], batch["v"], o_f, l_f, ws)
+    B.ckv_attend(shape, params, q_dec, k_out, v_out, o_c, l_c, ws, budgets=budgets, offsets=offsets)
+    quality["decode_check"] = {
+        "queries_per_head": n_dec, "mean_discarded_mass": float((1.0 - torch.exp(l_c - l_f).double()).clamp_min(0).mean()),
+        "mean_relative_output_error": float(((o_c - o_f).norm(dim=-1) / o_f.norm(dim=-1).clamp_min(1e-20)).mean()),
+        "what": "random N(0,1) decode queries attending over the compressed cache against the full cache"}
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         # a first unit gives the oracle's pace; then as many units as fit in about 15 s of wall time

@@ -139,6 +139,21 @@ ckv_status ckv_vnorm(const ckv_shape* shape, const ckv_params* params, const voi
                      float* scores_or_null, void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * Decode-side check of the compressed cache (the setting of Prop. 4.1; not part of the retention pass): softmax
+ * attention of n_dec decode queries per query head -- queries that come after the prompt and see every row -- over
+ *   compressed == 0: all L rows of k, v [Nu,Hkv,L,d] (strides of `shape`);
+ *   compressed == 1: the rows the pass kept; k, v are then k_out, v_out [Nu, Hkv min(B,L), d] and head g of unit u
+ *                    owns budgets[u,g] rows from row offsets[u,g].
+ * q_dec [Nu,H,n_dec,d] dense, in the dtype of `shape`; (H / Hkv) * n_dec <= 32, else CKV_ERR_UNSUPPORTED.
+ * out [Nu,H,n_dec,d] fp32 = softmax(q k^T / sqrt d) v;  lse [Nu,H,n_dec] fp32 = ln sum_t exp(q . k_t / sqrt d).
+ * With both runs, the discarded mass of the proposition is m = 1 - exp(lse_compressed - lse_full), the compressed
+ * output is the attention under the renormalised restriction p~, and |p - p~|_1 = 2 m.
+ */
+ckv_status ckv_attend(const ckv_shape* shape, const ckv_params* params, const void* q_dec, int32_t n_dec,
+                      const void* k, const void* v, int32_t compressed, const int32_t* budgets, const int32_t* offsets,
+                      float* out, float* lse, void* ws, size_t ws_bytes, void* stream);
+
+/*
  * Diagnostic of Prop. 4.1 on the observation-window rows (they stand in for decode queries): the attention mass
  * that survives the selection,
  *   kept[u,h,i] = sum over the retained positions t of KV head h/G that row i can see of A^h[n+i, t],

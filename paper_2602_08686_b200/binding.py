@@ -64,6 +64,7 @@ def lib() -> C.CDLL:
         L.ckv_select.argtypes = [shp, prm, fp, i32p, i32p, i32p, vp, sz, vp]
         L.ckv_vnorm.argtypes = [shp, prm, vp, fp, fp, vp, sz, vp]
         L.ckv_unit_max.argtypes = [shp, prm, fp, vp]
+        L.ckv_attend.argtypes = [shp, prm, vp, C.c_int32, vp, vp, C.c_int32, i32p, i32p, fp, fp, vp, sz, vp]
         L.ckv_kept_mass.argtypes = [shp, prm, vp, vp, i32p, i32p, i32p, fp, vp, sz, vp]
         L.ckv_prompt_mass.argtypes = [shp, prm, fp, fp, vp]
         L.ckv_global_scores.argtypes = [shp, prm, fp, fp, C.c_int32, fp, fp, vp]
@@ -79,7 +80,7 @@ def lib() -> C.CDLL:
         L.ckv_status_string.restype = C.c_char_p
         L.ckv_status_string.argtypes = [C.c_int]
         L.ckv_allocate_rows_host.argtypes = [C.c_int, C.c_int64, C.c_int64, C.c_int64, vp, vp]
-        for name in ("ckv_score", "ckv_score_noalloc", "ckv_budget", "ckv_select", "ckv_vnorm", "ckv_unit_max", "ckv_kept_mass", "ckv_prompt_mass", "ckv_global_scores", "ckv_gather", "ckv_compress", "ckv_compress_host",
+        for name in ("ckv_score", "ckv_score_noalloc", "ckv_budget", "ckv_select", "ckv_vnorm", "ckv_unit_max", "ckv_kept_mass", "ckv_attend", "ckv_prompt_mass", "ckv_global_scores", "ckv_gather", "ckv_compress", "ckv_compress_host",
                      "ckv_device_status", "ckv_version", "ckv_allocate_rows_host"):
             getattr(L, name).restype = C.c_int
         _lib = L
@@ -232,6 +233,15 @@ def ckv_global_scores(shape, params, head_w, pmass, units_total, scores, colmass
 def ckv_kept_mass(shape, params, q_win, k_out, indices, budgets, offsets, kept, ws, stream=None):
     _check(lib().ckv_kept_mass(C.byref(shape), C.byref(params), _ptr(q_win), _ptr(k_out), _ptr(indices), _ptr(budgets),
                                _ptr(offsets), _ptr(kept), _ptr(ws), ws.numel(), _stream(stream)), "ckv_kept_mass")
+
+
+def ckv_attend(shape, params, q_dec, k, v, out, lse, ws, budgets=None, offsets=None, stream=None):
+    """Attention of the decode queries q_dec [Nu,H,n_dec,d] over all rows of k, v, or over the gathered rows when
+    budgets and offsets are given."""
+    compressed = budgets is not None
+    _check(lib().ckv_attend(C.byref(shape), C.byref(params), _ptr(q_dec), int(q_dec.shape[2]), _ptr(k), _ptr(v),
+                            int(compressed), _ptr(budgets), _ptr(offsets), _ptr(out), _ptr(lse), _ptr(ws), ws.numel(),
+                            _stream(stream)), "ckv_attend")
 
 
 def ckv_unit_max(shape, params, scores, stream=None):

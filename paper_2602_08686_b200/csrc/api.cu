@@ -40,6 +40,11 @@ WsLayout ws_layout(const ckv_shape& s, const ckv_params& p) {
     w.bud_done = o, o = align_up(o + b.done_bytes);
   }
   w.pmass = o, o = align_up(o + (p.global_alpha ? Nu / (size_t)p.units_per_prompt * L * sizeof(float) : 0));
+  {
+    const size_t slots = Nu * Hkv * (size_t)attend_slices(s) * kAttendMaxRows;
+    w.att_ml = o, o = align_up(o + slots * sizeof(float2));
+    w.att_o = o, o = align_up(o + slots * kHeadDim * sizeof(float));
+  }
   w.vn_part = o, o = align_up(o + Nu * Hkv * ((L + kVnormRows - 1) / kVnormRows) * sizeof(float));
   w.vn_rho = o, o = align_up(o + (p.value_norm ? Nu * Hkv * L * sizeof(float) : 0));
   if (s.dtype == CKV_BF16) {
@@ -199,6 +204,23 @@ ckv_status ckv_vnorm(const ckv_shape* shape, const ckv_params* params, const voi
   float* part = reinterpret_cast<float*>((char*)ws + w.vn_part);
   CKV_CUDA(launch_vnorm_rows(*shape, v, rho, part, (cudaStream_t)stream));
   CKV_CUDA(launch_vnorm_finish(*shape, params->value_norm_eps, rho, part, scores_or_null, (cudaStream_t)stream));
+  return CKV_OK;
+}
+
+ckv_status ckv_attend(const ckv_shape* shape, const ckv_params* params, const void* q_dec, int32_t n_dec,
+                      const void* k, const void* v, int32_t compressed, const int32_t* budgets, const int32_t* offsets,
+                      float* out, float* lse, void* ws, size_t ws_bytes, void* stream) {
+  CKV_TRY(check_shape(shape));
+  CKV_TRY(check_params(shape, params));
+  if (n_dec < 1 || (shape->n_q_heads / shape->n_kv_heads) * n_dec > kAttendMaxRows) return CKV_ERR_UNSUPPORTED;
+  if (compressed != 0 && compressed != 1) return CKV_ERR_INVALID_ARG;
+  if (!all_aligned16({q_dec, k, v}) || !all_aligned4({out, lse})) return CKV_ERR_INVALID_ARG;
+  if (compressed && !all_aligned4({budgets, offsets})) return CKV_ERR_INVALID_ARG;
+  CKV_TRY(check_ws(shape, params, ws, ws_bytes));
+  const WsLayout w = ws_layout(*shape, *params);
+  char* base = (char*)ws;
+  CKV_CUDA(launch_attend(*shape, *params, q_dec, n_dec, k, v, compressed, budgets, offsets, out, lse, base + w.att_ml,
+                         base + w.att_o, (cudaStream_t)stream));
   return CKV_OK;
 }
 

@@ -12,6 +12,7 @@ constexpr int kMaxWindow = 64;
 constexpr int kMaxKvHeads = 64;
 constexpr int kPlainKeysPerBlock = 256;  // keys per CTA in the plain (SIMT) score kernels
 constexpr int kEntSpan = 512;            // positions per entropy partial of the budget stage
+constexpr int kAttendMaxRows = 32;       // query rows (group size x decode queries) of the decode-side check
 constexpr int kVnormRows = 256;          // value rows per block sum of the value-norm stage
 constexpr int kCountSpan = 8192;         // scores per counting CTA of the budget stage
 
@@ -35,6 +36,8 @@ struct WsLayout {
   size_t cnt_part; // int32 [Nu, Hkv, S]       candidate counts per slice
   size_t bud_done; // int32 [Nu]               CTAs of the unit that have finished counting
   size_t pmass;    // float [Nu / units_per_prompt, L] window mass summed over a prompt's units (only with global_alpha)
+  size_t att_ml;   // float2 [Nu, Hkv, slices, 32] and ...
+  size_t att_o;    // float [Nu, Hkv, slices, 32, 128]: per-slice partial results of the decode-side check
   size_t vn_part;  // float [Nu, Hkv, ceil(L / kVnormRows)] block sums of the value-row norms
   size_t vn_rho;   // float [Nu, Hkv, L]       value-norm ratios of the fused call (only with value_norm)
   size_t total;
@@ -126,6 +129,11 @@ cudaError_t launch_kept_mass(const ckv_shape& s, const ckv_params& p, const void
                              const int32_t* indices, const int32_t* budgets, const int32_t* offsets,
                              const void* stat_plain, const void* stat_tc, const int* marker, float* kept,
                              cudaStream_t st);
+// Decode-side check: attention of n_dec queries per head over all rows (compressed = 0) or the gathered rows.
+int attend_slices(const ckv_shape& s);
+cudaError_t launch_attend(const ckv_shape& s, const ckv_params& p, const void* q_dec, int n_dec, const void* k,
+                          const void* v, int compressed, const int32_t* budgets, const int32_t* offsets, float* out,
+                          float* lse, void* part_ml, void* part_o, cudaStream_t st);
 // Eq. 6 over all heads of a unit (the shared elastic selection): scores[u,g,:] <- max_g' scores[u,g',:].
 cudaError_t launch_unit_max(const ckv_shape& s, float* scores, cudaStream_t st);
 cudaError_t launch_select(const ckv_shape& s, const ckv_params& p, const float* scores, const int32_t* budgets,
