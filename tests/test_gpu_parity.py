@@ -520,3 +520,29 @@ def test_deterministic_run_to_run(B):
     c = B.compress(b["q"], b["k"], b["v"], b["head_w"], b["sens"], P, want_scores=True)
     for key in ("scores", "indices", "budgets", "k_out", "v_out", "entropy"):
         assert torch.equal(a[key], c[key]), key
+
+
+@pytest.mark.parametrize("run_tiles", [1, 3, 5, 64])
+def test_scan_run_size_does_not_change_the_result(B, run_tiles):
+    """The scan hands out its work in runs of key tiles; one tile per run (a single partial pair per run), sizes
+    that do not divide the tile count, and one run per chunk all give the oracle's scores and the same selection."""
+    cfg = gen.shrink(gen.CONFIGS["c2"], n_layers=3, seq_len=4500, budget_per_head=128, n_needles=8)
+    b = gen.make_batch(cfg, "cuda")
+    prob = problem_of(cfg, 3)
+    P = params_of(B, prob)
+    base = B.compress(b["q"], b["k"], b["v"], b["head_w"], b["sens"], P, want_scores=True)
+    prev_path = B.ckv_set_score_path(2)
+    prev = B.ckv_set_tunable("run_tiles", run_tiles)
+    try:
+        out = B.compress(b["q"], b["k"], b["v"], b["head_w"], b["sens"], P, want_scores=True)
+        assert B.ckv_device_status(out["ws"]) == B.OK
+    finally:
+        B.ckv_set_tunable("run_tiles", prev)
+        B.ckv_set_score_path(prev_path)
+    rel = ((out["scores"] - base["scores"]).abs() / base["scores"].abs().clamp_min(1e-20)).max().item()
+    assert rel < 1e-5, rel
+    sc, _ = oracle.score(prob, *(gen.as_numpy(b[x].cpu()) for x in ("q", "k", "head_w")))
+    gs = out["scores"].double().cpu().numpy()
+    assert (np.abs(gs - sc) / np.maximum(np.abs(sc), 1e-20)).max() <= SCORE_RTOL
+    idx, bud, off = (out[x].cpu().numpy() for x in ("indices", "budgets", "offsets"))
+    np.testing.assert_array_equal(idx, oracle.select(prob, gs, bud, off))
