@@ -546,3 +546,28 @@ def test_scan_run_size_does_not_change_the_result(B, run_tiles):
     assert (np.abs(gs - sc) / np.maximum(np.abs(sc), 1e-20)).max() <= SCORE_RTOL
     idx, bud, off = (out[x].cpu().numpy() for x in ("indices", "budgets", "offsets"))
     np.testing.assert_array_equal(idx, oracle.select(prob, gs, bud, off))
+
+
+def test_two_streams_two_work_spaces(B):
+    """Calls on different streams with their own work spaces do not disturb each other (the library keeps no
+    per-call global state)."""
+    cfgs = [gen.shrink(gen.CONFIGS["c2"], n_layers=2, seq_len=3000, budget_per_head=96, n_needles=4),
+            gen.shrink(gen.CONFIGS["c5"], n_layers=2, batch=1, seq_len=2100, budget_per_head=128, n_needles=4)]
+    batches = [gen.make_batch(c, "cuda") for c in cfgs]
+    Ps = [params_of(B, problem_of(c, 2)) for c in cfgs]
+    serial = [B.compress(b["q"], b["k"], b["v"], b["head_w"], b["sens"], P, want_scores=True) for b, P in zip(batches, Ps)]
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    outs = [[], []]
+    for rep in range(6):
+        for i in (0, 1):
+            b = batches[i]
+            with torch.cuda.stream(streams[i]):
+                outs[i].append(B.compress(b["q"], b["k"], b["v"], b["head_w"], b["sens"], Ps[i], want_scores=True,
+                                          stream=streams[i]))
+    torch.cuda.synchronize()
+    for i in (0, 1):
+        for o in outs[i]:
+            assert B.ckv_device_status(o["ws"]) == B.OK
+            for key in ("scores", "indices", "budgets", "k_out", "v_out"):
+                assert torch.equal(o[key], serial[i][key]), (i, key)
