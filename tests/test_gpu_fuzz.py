@@ -1,0 +1,71 @@
+"""Seeded random shapes and parameters: the fused GPU pass against the oracle's steps run on the GPU's own
+scores (exact for budgets and indices) and against the oracle's scores (tolerance), with the optional modes mixed in."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2602_08686_b200 import inputs as gen
+from test_gpu_parity import SCORE_RTOL, check_gather, params_of, problem_of
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2602_08686_b200 import binding
+    binding.lib()
+    assert torch.cuda.is_available()
+    return binding
+
+
+def draw(seed):
+    r = np.random.default_rng(seed)
+    Hkv = int(r.choice([1, 2, 3, 4, 8]))
+    G = int(r.choice([1, 2, 4, 7]))
+    W = int(r.choice([1, 5, 16, 32, 64]))
+    L = int(r.integers(max(W + 40, 130), 2600))
+    dtype = str(r.choice(["bf16", "bf16", "f32"]))
+    pool_kind = int(r.choice([0, 1, 1, 2]))
+    pool_size = 1 if pool_kind == 0 else int(r.choice([1, 3, 5, 7, 15]))
+    budget = int(r.integers(W + 8, min(L + 50, W + 400)))
+    n = L - W
+    floor = int(r.integers(0, max(1, min(9, budget - W)))) if budget < L else 0
+    layers = int(r.integers(1, 4)) * 2
+    modes = dict(value_norm=bool(r.integers(0, 2)), shared_elastic=bool(r.integers(0, 4) == 0),
+                 global_alpha=bool(r.integers(0, 4) == 0), units_per_prompt=2)
+    cfg = gen.shrink(gen.CONFIGS["c2"], config_id=100 + seed, n_layers=layers, batch=1, n_q_heads=Hkv * G, n_kv_heads=Hkv,
+                     seq_len=L, window=W, pool_kind=pool_kind, pool_size=pool_size, budget_per_head=budget,
+                     floor_per_head=floor, n_needles=2 if n > 64 else 0, dtype=dtype, n_buckets=int(r.choice([1, 7, 16])))
+    return cfg, modes
+
+
+@pytest.mark.parametrize("seed", range(100))
+def test_random_case(B, seed):
+    cfg, modes = draw(seed)
+    Nu = cfg.n_units
+    b = gen.make_batch(cfg, "cpu")
+    # thresholds near the bulk of the scores, so that the candidate counts differ between heads
+    prob = problem_of(cfg, Nu, **modes)
+    qn, kn, vn, hw = (gen.as_numpy(b[x]) for x in ("q", "k", "v", "head_w"))
+    sc, cm = oracle.score(prob, qn, kn, hw, v=vn if modes["value_norm"] else None)
+    qs = np.quantile(sc, np.linspace(0.3, 0.995, cfg.n_buckets)).astype(np.float32)
+    sens = torch.from_numpy(qs[np.random.default_rng(seed).permutation(cfg.n_buckets)].copy())
+    P = params_of(B, prob)
+    for f in ("value_norm", "shared_elastic", "global_alpha", "units_per_prompt"):
+        setattr(P, f, modes[f])
+    out = B.compress(*(b[x].cuda() for x in ("q", "k", "v", "head_w")), sens.cuda(), P, want_scores=True)
+    assert B.ckv_device_status(out["ws"]) == B.OK
+    gs = out["scores"].double().cpu().numpy()
+    rel = np.abs(gs - sc) / np.maximum(np.abs(sc), 1e-20)
+    assert rel.max() <= SCORE_RTOL, (rel.max(), cfg, modes)
+    idx, bud, off = (out[x].cpu().numpy() for x in ("indices", "budgets", "offsets"))
+    bucket = out["bucket"].cpu().numpy()
+    for u in range(Nu):
+        prob_u = problem_of(cfg, 1, bucket_override=int(bucket[u]), shared_elastic=modes["shared_elastic"])
+        mine = oracle.budget(prob_u, gs[u:u + 1], cm[u:u + 1], sens.numpy())
+        assert (mine["budgets"][0] == bud[u]).all(), (u, mine["budgets"], bud[u], cfg, modes)
+    want = oracle.select(prob, gs, bud, off)
+    for u in range(Nu):
+        np.testing.assert_array_equal(idx[u, :off[u, -1]], want[u, :off[u, -1]])
+    check_gather(b["k"], b["v"], out["k_out"], out["v_out"], idx, off, prob)
