@@ -69,3 +69,25 @@ def test_random_case(B, seed):
     for u in range(Nu):
         np.testing.assert_array_equal(idx[u, :off[u, -1]], want[u, :off[u, -1]])
     check_gather(b["k"], b["v"], out["k_out"], out["v_out"], idx, off, prob)
+
+
+def draw_long(seed):
+    r = np.random.default_rng(1000 + seed)
+    Hkv, G = int(r.choice([1, 2])), int(r.choice([1, 4, 7]))
+    W = int(r.choice([16, 32, 64]))
+    L = int(r.integers(30000, 80000))
+    pool_kind = int(r.choice([1, 2]))
+    cfg = gen.shrink(gen.CONFIGS["c4" if seed % 2 else "c2"], config_id=200 + seed, n_layers=2, batch=1,
+                     n_q_heads=Hkv * G, n_kv_heads=Hkv, seq_len=L, window=W, pool_kind=pool_kind,
+                     pool_size=int(r.choice([3, 7])), budget_per_head=int(r.integers(W + 64, 3000)),
+                     floor_per_head=int(r.integers(0, 9)), n_needles=8)
+    modes = dict(value_norm=bool(r.integers(0, 2)), shared_elastic=False, global_alpha=bool(r.integers(0, 3) == 0),
+                 units_per_prompt=2)
+    return cfg, modes
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_random_long_case(B, seed, monkeypatch):
+    """The same at lengths that take the selection's cluster paths and many key tiles per chunk."""
+    monkeypatch.setattr("test_gpu_fuzz.draw", lambda s: draw_long(s))
+    test_random_case(B, seed)
