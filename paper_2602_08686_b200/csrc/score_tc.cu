@@ -31,6 +31,7 @@
 #include <cuda_bf16.h>
 
 #include <atomic>
+#include <type_traits>
 #include <string>
 
 #include "ckv_common.cuh"
@@ -789,23 +790,29 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
 #pragma unroll
           for (int hh = 0; hh < kHeadsPerSlice; ++hh) acc2[hh] = pack2(0.f, 0.f);
           const uint64_t scale2 = pack2(kScale, kScale);
+          // the slice's exponentials; the causal test of the window keys only exists in the copy for the tiles
+          // that reach past the prefix, so that the common copy is straight-line code
+          auto slice = [&](auto masked) {
 #pragma unroll
-          for (int j4 = 0; j4 < 8; ++j4) {
-            const float4 b4 = reinterpret_cast<const float4*>(nb)[cc * 8 + j4];
-            const uint64_t bb2[2] = {pack2(b4.x, b4.y), pack2(b4.z, b4.w)};
+            for (int j4 = 0; j4 < 8; ++j4) {
+              const float4 b4 = reinterpret_cast<const float4*>(nb)[cc * 8 + j4];
+              const uint64_t bb2[2] = {pack2(b4.x, b4.y), pack2(b4.z, b4.w)};
 #pragma unroll
-            for (int e2 = 0; e2 < 2; ++e2) {
-              const int jj = j4 * 4 + 2 * e2;
-              float x0, x1;
-              unpack2(fma2(pack2(v[jj], v[jj + 1]), scale2, bb2[e2]), x0, x1);
-              float p0 = ex2(x0), p1 = ex2(x1);
-              if (tail) {
-                if (t > a.n + (cc * 32 + jj) % W) p0 = 0.f;
-                if (t > a.n + (cc * 32 + jj + 1) % W) p1 = 0.f;
+              for (int e2 = 0; e2 < 2; ++e2) {
+                const int jj = j4 * 4 + 2 * e2;
+                float x0, x1;
+                unpack2(fma2(pack2(v[jj], v[jj + 1]), scale2, bb2[e2]), x0, x1);
+                float p0 = ex2(x0), p1 = ex2(x1);
+                if constexpr (decltype(masked)::value) {
+                  if (t > a.n + (cc * 32 + jj) % W) p0 = 0.f;
+                  if (t > a.n + (cc * 32 + jj + 1) % W) p1 = 0.f;
+                }
+                acc2[W >= 32 ? 0 : jj / W] = add2(acc2[W >= 32 ? 0 : jj / W], pack2(p0, p1));
               }
-              acc2[W >= 32 ? 0 : jj / W] = add2(acc2[W >= 32 ? 0 : jj / W], pack2(p0, p1));
             }
-          }
+          };
+          if (tail) slice(std::true_type{});
+          else slice(std::false_type{});
           float acc[kHeadsPerSlice][2];
 #pragma unroll
           for (int hh = 0; hh < kHeadsPerSlice; ++hh) unpack2(acc2[hh], acc[hh][0], acc[hh][1]);
