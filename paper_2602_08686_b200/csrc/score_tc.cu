@@ -382,7 +382,8 @@ __device__ __forceinline__ bool wait_flag(Pred pred, unsigned sleep_ns, volatile
   return true;
 }
 
-template <int W>
+// kGrouped: pass 2 writes the per-group maximum and mass (TcArgs::zgrp) instead of per-head column sums.
+template <int W, bool kGrouped>
 __global__ void __launch_bounds__(kThreads, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map, TcArgs a) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -763,7 +764,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         const float* nb = sm.nbias[d.nbias_buf];
         constexpr int kHeadsPerSlice = W >= 32 ? 1 : 32 / W;  // heads inside one 32-row TMEM load
         float* out = a.csum + (int64_t)d.head0 * a.L + t;
-        const bool grouped = a.zgrp != nullptr;
+        constexpr bool grouped = kGrouped;
         const float* hw = a.head_w + d.part_slot;
         float wv[4] = {0.f, 0.f, 0.f, 0.f};   // the block's head weights when it holds at most four heads
         if (grouped && W >= 32) {
@@ -891,10 +892,11 @@ cuuint64_t legal_stride(uint64_t extent, int64_t stride_elems, cuuint64_t fallba
   return (extent == 1 || stride_elems <= 0) ? fallback_bytes : (cuuint64_t)stride_elems * 2;
 }
 
-template <int W>
-cudaError_t launch_w(const CUtensorMap& qm, const CUtensorMap& km, const TcArgs& a, int grid, cudaStream_t st) {
+template <int W, bool kGrouped>
+cudaError_t launch_wg(const CUtensorMap& qm, const CUtensorMap& km, const TcArgs& a, int grid, cudaStream_t st) {
   const size_t smem = sizeof(Smem);
-  cudaError_t e = cudaFuncSetAttribute(score_tc_kernel<W>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  auto kernel = score_tc_kernel<W, kGrouped>;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid), cfg.blockDim = dim3(kThreads), cfg.dynamicSmemBytes = smem, cfg.stream = st;
@@ -902,7 +904,11 @@ cudaError_t launch_w(const CUtensorMap& qm, const CUtensorMap& km, const TcArgs&
   attr[0].id = cudaLaunchAttributeCooperative;
   attr[0].val.cooperative = 1;  // all CTAs co-resident: CTAs wait on flags other CTAs set
   cfg.attrs = attr, cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, score_tc_kernel<W>, qm, km, a);
+  return cudaLaunchKernelEx(&cfg, kernel, qm, km, a);
+}
+template <int W>
+cudaError_t launch_w(const CUtensorMap& qm, const CUtensorMap& km, const TcArgs& a, int grid, cudaStream_t st) {
+  return a.zgrp ? launch_wg<W, true>(qm, km, a, grid, st) : launch_wg<W, false>(qm, km, a, grid, st);
 }
 
 }  // namespace
