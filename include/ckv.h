@@ -280,7 +280,7 @@ int ckv_set_score_path(int path);
 void ckv_set_scan_events(void* start_event, void* stop_event);
 
 /* Diagnostic knobs of the tensor-core scan (process-wide; the scores do not depend on them):
- *   "run_tiles"      key tiles per run, the unit CTAs take work in (1..64, default 8);
+ *   "run_tiles"      key tiles per run, the unit CTAs take work in (1..64, default 16);
  *   "l2_hints"       1 (default): first-pass K loads ask L2 to keep their lines and second-pass loads
  *                    release them; 0: no hints;
  *   "group_fuse"     1 (default): where a KV group's query heads fill one 128-row block and the pooling

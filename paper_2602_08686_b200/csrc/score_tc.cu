@@ -62,7 +62,7 @@ constexpr float kScale = 0.12751743074602467f;
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 
 // Tunables of the schedule (process-wide; see ckv_set_tunable).
-std::atomic<int> g_run_tiles{8};        // key tiles per run
+std::atomic<int> g_run_tiles{16};       // key tiles per run
 std::atomic<int> g_l2_hints{1};         // 1: P1 loads keep their lines (evict_last), P2 loads release them
 
 struct TcArgs {
