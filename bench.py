@@ -291,6 +291,23 @@ def main():
                                "frac": (k2_bytes + gather_bytes) / (ms_per_step * 1e-3) / 1e9 / peak,
                                "frac_of_nominal_8TBs": (k2_bytes + gather_bytes) / (ms_per_step * 1e-3) / 8e12},
                 "stage_ms": stage_ms}
+    # The scan's other ceiling: one ex2 per (query row, key) and pass on the special-function unit, 16 per clock and SM.
+    n_exp = 2.0 * n_units * cfg.n_q_heads * cfg.window * L
+    sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
+    sm_max_mhz = (clocks or {}).get("sm_max_mhz") or 1965.0
+    exp_peak = 16.0 * sm_count * sm_max_mhz * 1e6 / 1e9          # G exp/s at the maximum SM clock
+    exp_rate = n_exp / (scan_ms * 1e-3) / 1e9
+    alu = {"bound": "alu", "what": "ex2.approx on the special-function unit: 2*H*W*L per unit, 16 per clock and SM "
+                                   "at the maximum SM clock",
+           "achieved": exp_rate, "peak": exp_peak, "unit": "Gexp/s", "frac": exp_rate / exp_peak}
+    if alu["frac"] > roofline["frac"]:      # many query rows per key byte: the exponentials bind, not HBM
+        hbm = {k_: roofline[k_] for k_ in ("bound", "achieved", "peak", "peak_kind", "unit", "frac")}
+        roofline.update({k_: alu[k_] for k_ in ("bound", "achieved", "peak", "unit", "frac")})
+        roofline["peak_kind"] = "derived: 16 ex2 per clock per SM x SMs x maximum SM clock"
+        roofline["what"] = alu["what"]
+        roofline["hbm"] = hbm
+    else:
+        roofline["alu"] = alu
 
     # ---- end to end through ckv_compress_host (pinned host buffers, copies inside the timed region) ----
     e2e = None
