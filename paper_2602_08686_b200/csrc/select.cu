@@ -53,143 +53,173 @@ __device__ __forceinline__ void transpose32(uint32_t (&a)[32]) {
   }
 }
 
+// 4-byte asynchronous copy into shared memory; src_bytes 0 writes zeros and reads nothing.
+__device__ __forceinline__ void async_copy4(uint32_t* dst, const float* src, int src_bytes) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src),
+               "r"(src_bytes)
+               : "memory");
+}
+__device__ __forceinline__ void async_copy_wait() {
+  asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+}
+
 // kCluster CTAs of one thread-block cluster share a head: CTA r holds the positions from r * kSlicedMax.
 // Every warp then sends its counts to all CTAs of the cluster through distributed shared memory and the
-// step's barrier spans the cluster.
+// step's barrier spans the cluster.  A CTA (cluster) takes the heads blockIdx.x / kCluster, + stride, ...;
+// the scores of its next head stream into the staging area while it searches the current one.
 template <int kCluster>
 __global__ void __launch_bounds__(kThreads) select_sliced_kernel(ckv_shape s, int64_t unit_rows,
                                                                  const float* __restrict__ scores,
                                                                  const int32_t* __restrict__ budgets,
                                                                  const int32_t* __restrict__ offsets,
                                                                  int32_t* __restrict__ indices) {
-  extern __shared__ __align__(16) uint32_t stage[];   // [warps in use][1024] keys in position order
+  extern __shared__ __align__(16) uint32_t stage[];   // [warps in use][1024] score bits in position order
   __shared__ uint2 wcnt[2][kCluster][kWarps];
   __shared__ uint32_t wtot[kWarps];
   __shared__ uint32_t ctot[kCluster];
   pdl_launch_dependents();
   pdl_wait();   // budgets, offsets and scores come from the kernels before
   const int Hkv = s.n_kv_heads, W = s.window, n = s.seq_len - W;
-  const int head = blockIdx.x / kCluster, rank = blockIdx.x % kCluster;
-  const int u = head / Hkv, g = head % Hkv;
-  const int e = budgets[(int64_t)u * Hkv + g] - W;
-  int32_t* out = indices + (int64_t)u * unit_rows + offsets[(int64_t)u * (Hkv + 1) + g];
-  const float* sc = scores + ((int64_t)u * Hkv + g) * n;
+  const int n_heads = s.n_units * Hkv, stride = (int)gridDim.x / kCluster;
+  const int rank = blockIdx.x % kCluster;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int cbase = rank * kSlicedMax;                      // first position of this CTA
   const int first = cbase + 32 * (int)threadIdx.x;          // first position of this thread
-
-  // the branches below are taken by all CTAs of a cluster alike
-  if (rank == 0)
-    for (int i = threadIdx.x; i < W; i += kThreads) out[e + i] = n + i;
-  if (e <= 0) return;
-  if (e >= n) {
-    for (int t = cbase + threadIdx.x; t < min(n, cbase + kSlicedMax); t += kThreads) out[t] = t;
-    return;
-  }
+  const int wbase = warp * 1024;                            // first position of the warp inside the CTA
+  const bool staged = cbase + wbase < n;                    // the warp holds positions of the prefix
+  uint32_t* const ws = stage + wbase;
   auto step_barrier = [&]() {
     if constexpr (kCluster == 1) __syncthreads();
     else cooperative_groups::this_cluster().sync();
   };
-
-  // a[31 - k] = key of position first + (k + 4 * lane) % 32: the 16-byte pieces of the thread's line are
-  // fetched in an order rotated by the lane so that a quarter warp touches every bank once
-  uint32_t a[32];
-  const int wbase = warp * 1024;
-  if (cbase + wbase < n) {
-    uint32_t* ws = stage + wbase;
+  // every warp copies its own 1024 scores: nothing but the warp reads them
+  auto prefetch = [&](int head) {
+    if (!staged) return;
+    const float* sc = scores + (int64_t)head * n;
 #pragma unroll
     for (int j = 0; j < 32; ++j) {
       const int t = cbase + wbase + 32 * j + lane;
-      ws[32 * j + lane] = t < n ? key_of(sc[t]) : 0u;
+      async_copy4(ws + 32 * j + lane, t < n ? sc + t : sc, t < n ? 4 : 0);
     }
-    __syncwarp();
-    const uint4* line = reinterpret_cast<const uint4*>(ws + 32 * lane);
-#pragma unroll
-    for (int q = 0; q < 8; ++q) {
-      const uint4 v = line[(q + lane) & 7];
-      a[31 - 4 * q] = v.x, a[30 - 4 * q] = v.y, a[29 - 4 * q] = v.z, a[28 - 4 * q] = v.w;
-    }
-  } else {
-#pragma unroll
-    for (int k = 0; k < 32; ++k) a[k] = 0u;
-  }
-  transpose32(a);   // a[31 - b] bit k = bit b of the k-th fetched key
-
+  };
   // positions of the thread that exist, in fetch order (bit k <-> position first + (k + 4 lane) % 32)
   const int rot = (4 * lane) & 31;
   const int have = min(max(n - first, 0), 32);
   const uint32_t valid_pos = have >= 32 ? 0xffffffffu : ((1u << have) - 1u);
-  uint32_t alive = __funnelshift_r(valid_pos, valid_pos, rot);   // keys equal to the decided bits so far
-  uint32_t gt = 0u;                                              // keys above the k-th
-  int above = 0;                                                 // their number over the whole head
+
+  int head = blockIdx.x / kCluster;
+  if (head < n_heads) prefetch(head);
+  // the branches below are taken by all CTAs of a cluster alike
+  for (; head < n_heads; head += stride) {
+    const int u = head / Hkv, g = head - u * Hkv;
+    const int e = budgets[(int64_t)u * Hkv + g] - W;
+    int32_t* out = indices + (int64_t)u * unit_rows + offsets[(int64_t)u * (Hkv + 1) + g];
+
+    // a[31 - k] = key of position first + (k + 4 * lane) % 32: the 16-byte pieces of the thread's line are
+    // fetched in an order rotated by the lane so that a quarter warp touches every bank once
+    uint32_t a[32];
+    async_copy_wait();
+    __syncwarp();
+    if (staged) {
+      const uint4* line = reinterpret_cast<const uint4*>(ws + 32 * lane);
 #pragma unroll
-  for (int st = 0; st < 16; ++st) {
-    const uint32_t p1 = a[2 * st], p0 = a[2 * st + 1];   // planes of bits 31 - 2 st and 30 - 2 st
-    const uint32_t h = alive & p1, l = alive & ~p1;
-    const uint32_t h1 = h & p0, l1 = l & p0;
-    const uint32_t r1 = __reduce_add_sync(0xffffffffu, (uint32_t)__popc(h1) | ((uint32_t)__popc(h) << 16));
-    const uint32_t r2 = __reduce_add_sync(0xffffffffu, (uint32_t)__popc(l1));
-    // the other buffer is written in the next step, this one again only after that step's barrier
-    if constexpr (kCluster == 1) {
-      if (lane == 0) wcnt[st & 1][0][warp] = make_uint2(r1, r2);
+      for (int q = 0; q < 8; ++q) {
+        const uint4 v = line[(q + lane) & 7];
+        a[31 - 4 * q] = key_of(__uint_as_float(v.x)), a[30 - 4 * q] = key_of(__uint_as_float(v.y));
+        a[29 - 4 * q] = key_of(__uint_as_float(v.z)), a[28 - 4 * q] = key_of(__uint_as_float(v.w));
+      }
     } else {
-      if (lane < kCluster)
-        *cooperative_groups::this_cluster().map_shared_rank(&wcnt[st & 1][rank][warp], lane) = make_uint2(r1, r2);
-    }
-    step_barrier();
-    uint32_t wx = 0, wy = 0;   // lane l adds warp l of every CTA: both 16-bit fields stay below 2^14
 #pragma unroll
-    for (int c = 0; c < kCluster; ++c) {
-      const uint2 w = wcnt[st & 1][c][lane];
-      wx += w.x, wy += w.y;
+      for (int k = 0; k < 32; ++k) a[k] = 0u;
     }
-    int t11, t1x;
-    if constexpr (kCluster == 1) {
-      const uint32_t t1 = __reduce_add_sync(0xffffffffu, wx);
-      t11 = (int)(t1 & 0xffffu), t1x = (int)(t1 >> 16);
-    } else {
-      t11 = (int)__reduce_add_sync(0xffffffffu, wx & 0xffffu), t1x = (int)__reduce_add_sync(0xffffffffu, wx >> 16);
+    __syncwarp();   // the warp has read its lines: the next head's scores may overwrite them
+    if (head + stride < n_heads) prefetch(head + stride);
+
+    if (rank == 0)
+      for (int i = threadIdx.x; i < W; i += kThreads) out[e + i] = n + i;
+    if (e <= 0) continue;
+    if (e >= n) {
+      for (int t = cbase + threadIdx.x; t < min(n, cbase + kSlicedMax); t += kThreads) out[t] = t;
+      continue;
     }
-    const int t01 = (int)__reduce_add_sync(0xffffffffu, wy);
-    if (above + t11 >= e) {               // digit 11
-      alive = h1;
-    } else if (above + t1x >= e) {        // digit 10
-      gt |= h1, above += t11, alive = h & ~p0;
-    } else if (above + t1x + t01 >= e) {  // digit 01
-      gt |= h, above += t1x, alive = l1;
-    } else {                              // digit 00
-      gt |= h | l1, above += t1x + t01, alive = l & ~p0;
-    }
-  }
-  // alive: keys equal to the k-th; the lowest (e - above) positions among them are kept
-  const int want = e - above;
-  const uint32_t gtp = __funnelshift_l(gt, gt, rot), eqp = __funnelshift_l(alive, alive, rot);   // position order
-  const uint32_t mine = (uint32_t)__popc(gtp) | ((uint32_t)__popc(eqp) << 16);
-  uint32_t incl = mine;
+    transpose32(a);   // a[31 - b] bit k = bit b of the k-th fetched key
+
+    uint32_t alive = __funnelshift_r(valid_pos, valid_pos, rot);   // keys equal to the decided bits so far
+    uint32_t gt = 0u;                                              // keys above the k-th
+    int above = 0;                                                 // their number over the whole head
+    int tied = n;                                                  // keys of the whole head still in `alive`
 #pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const uint32_t x = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += x;
-  }
-  if (lane == 31) wtot[warp] = incl;
-  __syncthreads();
-  const uint32_t wt = wtot[lane];
-  const uint32_t before = __reduce_add_sync(0xffffffffu, lane < warp ? wt : 0u) + incl - mine;
-  int gt_before = (int)(before & 0xffffu), eq_before = (int)(before >> 16);
-  if constexpr (kCluster > 1) {   // kept keys of the CTAs holding lower positions
-    const uint32_t total = __reduce_add_sync(0xffffffffu, wt);
-    if (warp == 0 && lane < kCluster) *cooperative_groups::this_cluster().map_shared_rank(&ctot[rank], lane) = total;
-    cooperative_groups::this_cluster().sync();
-    for (int c = 0; c < rank; ++c) gt_before += (int)(ctot[c] & 0xffffu), eq_before += (int)(ctot[c] >> 16);
-  }
-  uint32_t m = gtp | eqp;
-  while (m) {
-    const int j = __ffs((int)m) - 1;
-    const uint32_t bit = 1u << j;
-    m &= m - 1u;
-    const int gb = gt_before + __popc(gtp & (bit - 1u)), eb = eq_before + __popc(eqp & (bit - 1u));
-    if (gtp & bit) out[gb + min(eb, want)] = first + j;
-    else if (eb < want) out[gb + eb] = first + j;
+    for (int st = 0; st < 16; ++st) {
+      const uint32_t p1 = a[2 * st], p0 = a[2 * st + 1];   // planes of bits 31 - 2 st and 30 - 2 st
+      const uint32_t h = alive & p1, l = alive & ~p1;
+      const uint32_t h1 = h & p0, l1 = l & p0;
+      const uint32_t r1 = __reduce_add_sync(0xffffffffu, (uint32_t)__popc(h1) | ((uint32_t)__popc(h) << 16));
+      const uint32_t r2 = __reduce_add_sync(0xffffffffu, (uint32_t)__popc(l1));
+      // the other buffer is written in the next step, this one again only after that step's barrier
+      if constexpr (kCluster == 1) {
+        if (lane == 0) wcnt[st & 1][0][warp] = make_uint2(r1, r2);
+      } else {
+        if (lane < kCluster)
+          *cooperative_groups::this_cluster().map_shared_rank(&wcnt[st & 1][rank][warp], lane) = make_uint2(r1, r2);
+      }
+      step_barrier();
+      uint32_t wx = 0, wy = 0;   // lane l adds warp l of every CTA: both 16-bit fields stay below 2^14
+#pragma unroll
+      for (int c = 0; c < kCluster; ++c) {
+        const uint2 w = wcnt[st & 1][c][lane];
+        wx += w.x, wy += w.y;
+      }
+      int t11, t1x;
+      if constexpr (kCluster == 1) {
+        const uint32_t t1 = __reduce_add_sync(0xffffffffu, wx);
+        t11 = (int)(t1 & 0xffffu), t1x = (int)(t1 >> 16);
+      } else {
+        t11 = (int)__reduce_add_sync(0xffffffffu, wx & 0xffffu), t1x = (int)__reduce_add_sync(0xffffffffu, wx >> 16);
+      }
+      const int t01 = (int)__reduce_add_sync(0xffffffffu, wy);
+      if (above + t11 >= e) {               // digit 11
+        alive = h1, tied = t11;
+      } else if (above + t1x >= e) {        // digit 10
+        gt |= h1, above += t11, alive = h & ~p0, tied = t1x - t11;
+      } else if (above + t1x + t01 >= e) {  // digit 01
+        gt |= h, above += t1x, alive = l1, tied = t01;
+      } else {                              // digit 00
+        gt |= h | l1, above += t1x + t01, alive = l & ~p0, tied -= t1x + t01;
+      }
+      // every key that still matches is kept: the lower bits decide nothing (the same test in every thread
+      // of the cluster, so all leave together)
+      if (above + tied == e) break;
+    }
+    // alive: keys equal to the k-th; the lowest (e - above) positions among them are kept
+    const int want = e - above;
+    const uint32_t gtp = __funnelshift_l(gt, gt, rot), eqp = __funnelshift_l(alive, alive, rot);   // position order
+    const uint32_t mine = (uint32_t)__popc(gtp) | ((uint32_t)__popc(eqp) << 16);
+    uint32_t incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t x = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += x;
+    }
+    if (lane == 31) wtot[warp] = incl;
+    __syncthreads();
+    const uint32_t wt = wtot[lane];
+    const uint32_t before = __reduce_add_sync(0xffffffffu, lane < warp ? wt : 0u) + incl - mine;
+    int gt_before = (int)(before & 0xffffu), eq_before = (int)(before >> 16);
+    if constexpr (kCluster > 1) {   // kept keys of the CTAs holding lower positions
+      const uint32_t total = __reduce_add_sync(0xffffffffu, wt);
+      if (warp == 0 && lane < kCluster) *cooperative_groups::this_cluster().map_shared_rank(&ctot[rank], lane) = total;
+      cooperative_groups::this_cluster().sync();
+      for (int c = 0; c < rank; ++c) gt_before += (int)(ctot[c] & 0xffffu), eq_before += (int)(ctot[c] >> 16);
+    }
+    uint32_t m = gtp | eqp;
+    while (m) {
+      const int j = __ffs((int)m) - 1;
+      const uint32_t bit = 1u << j;
+      m &= m - 1u;
+      const int gb = gt_before + __popc(gtp & (bit - 1u)), eb = eq_before + __popc(eqp & (bit - 1u));
+      if (gtp & bit) out[gb + min(eb, want)] = first + j;
+      else if (eb < want) out[gb + eb] = first + j;
+    }
   }
 }
 
@@ -342,7 +372,6 @@ cudaError_t launch_sliced(const ckv_shape& s, int n, int64_t unit_rows, const fl
                                        kSlicedMax * (int)sizeof(uint32_t));
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3((unsigned)(s.n_units * s.n_kv_heads * kCluster));
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = kCluster == 1 ? smem : kSlicedMax * sizeof(uint32_t);
   cfg.stream = st;
@@ -351,6 +380,25 @@ cudaError_t launch_sliced(const ckv_shape& s, int n, int64_t unit_rows, const fl
   attr[0].val.clusterDim.x = kCluster, attr[0].val.clusterDim.y = 1, attr[0].val.clusterDim.z = 1;
   attr[1] = pdl_attribute();
   cfg.attrs = attr, cfg.numAttrs = 2;
+  // as many CTAs (clusters) as the device holds at once; each loops over its share of the heads
+  static int resident = 0;   // one CTA of this kernel fills an SM: the answer depends on the device only
+  if (resident == 0) {
+    int dev = 0, sms = 0, clusters = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    clusters = sms / kCluster;
+    if (kCluster > 1) {
+      cfg.gridDim = dim3((unsigned)(sms / kCluster * kCluster));
+      int active = 0;
+      if (cudaOccupancyMaxActiveClusters(&active, select_sliced_kernel<kCluster>, &cfg) == cudaSuccess && active > 0)
+        clusters = active;
+      else
+        (void)cudaGetLastError();
+    }
+    resident = clusters > 0 ? clusters : 1;
+  }
+  const int n_heads = s.n_units * s.n_kv_heads;
+  cfg.gridDim = dim3((unsigned)(std::min(n_heads, resident) * kCluster));
   return cudaLaunchKernelEx(&cfg, select_sliced_kernel<kCluster>, s, unit_rows, scores, budgets, offsets, indices);
 }
 
