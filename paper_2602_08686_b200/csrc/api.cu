@@ -272,7 +272,8 @@ ckv_status ckv_select(const ckv_shape* shape, const ckv_params* params, const fl
   CKV_TRY(check_params(shape, params));
   if (!all_aligned4({scores, budgets, offsets, indices})) return CKV_ERR_INVALID_ARG;
   CKV_TRY(check_ws(shape, params, ws, ws_bytes));
-  CKV_CUDA(launch_select(*shape, *params, scores, budgets, offsets, indices, (cudaStream_t)stream));
+  int* status = reinterpret_cast<int*>(static_cast<char*>(ws) + ws_layout(*shape, *params).status);
+  CKV_CUDA(launch_select(*shape, *params, scores, budgets, offsets, indices, status, (cudaStream_t)stream));
   return CKV_OK;
 }
 
@@ -321,7 +322,7 @@ ckv_status ckv_compress(const ckv_shape* shape, const ckv_params* params, const 
   if (params->shared_elastic) CKV_CUDA(launch_unit_max(*shape, scores, st));
   CKV_CUDA(launch_budget(*shape, *params, scores, sens, budgets, offsets, bucket, entropy, base + w.ent_part,
                          base + w.cnt_part, base + w.bud_done, st));
-  CKV_CUDA(launch_select(*shape, *params, scores, budgets, offsets, indices, st));
+  CKV_CUDA(launch_select(*shape, *params, scores, budgets, offsets, indices, reinterpret_cast<int*>(base + w.status), st));
   CKV_CUDA(launch_gather(*shape, *params, k, v, indices, offsets, k_out, v_out, st));
   return CKV_OK;
 }

@@ -137,7 +137,7 @@ cudaError_t launch_attend(const ckv_shape& s, const ckv_params& p, const void* q
 // Eq. 6 over all heads of a unit (the shared elastic selection): scores[u,g,:] <- max_g' scores[u,g',:].
 cudaError_t launch_unit_max(const ckv_shape& s, float* scores, cudaStream_t st);
 cudaError_t launch_select(const ckv_shape& s, const ckv_params& p, const float* scores, const int32_t* budgets,
-                          const int32_t* offsets, int32_t* indices, cudaStream_t st);
+                          const int32_t* offsets, int32_t* indices, int* status, cudaStream_t st);
 cudaError_t launch_gather(const ckv_shape& s, const ckv_params& p, const void* k, const void* v,
                           const int32_t* indices, const int32_t* offsets, void* k_out, void* v_out,
                           cudaStream_t st);

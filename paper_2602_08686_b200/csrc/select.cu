@@ -63,21 +63,73 @@ __device__ __forceinline__ void async_copy_wait() {
   asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
 }
 
+// Exchange of a search step's counts between the CTAs of a cluster: every warp sends its two words to each
+// CTA with one asynchronous store that also credits the receiver's transaction barrier, so a step costs
+// one trip across the cluster instead of a store and a cluster-wide barrier.
+__device__ __forceinline__ uint32_t cluster_address(const void* local, int cta) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"((uint32_t)__cvta_generic_to_shared(local)), "r"(cta));
+  return r;
+}
+__device__ __forceinline__ void barrier_init(uint64_t* bar, int arrivals) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"((uint32_t)__cvta_generic_to_shared(bar)), "r"(arrivals) : "memory");
+}
+__device__ __forceinline__ void barrier_expect(uint64_t* bar, int bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"((uint32_t)__cvta_generic_to_shared(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void store_credit(uint32_t dst, uint64_t v, uint32_t bar) {
+  asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.b64 [%0], %1, [%2];" ::"r"(dst), "l"(v), "r"(bar) : "memory");
+}
+__device__ __forceinline__ bool barrier_test(uint64_t* bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(done)
+      : "r"((uint32_t)__cvta_generic_to_shared(bar)), "r"(parity)
+      : "memory");
+  return done != 0;
+}
+// Waits for the phase with the given parity, for two seconds at most.
+__device__ __forceinline__ bool barrier_wait_bounded(uint64_t* bar, uint32_t parity) {
+  if (barrier_test(bar, parity)) return true;
+  unsigned long long t0, t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i)
+      if (barrier_test(bar, parity)) return true;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    if (t - t0 > 2000000000ull) return false;
+  }
+}
+constexpr int kSelectTimeoutCode = 51;   // status word: a cluster exchange of the selection gave up
+
 // kCluster CTAs of one thread-block cluster share a head: CTA r holds the positions from r * kSlicedMax.
-// Every warp then sends its counts to all CTAs of the cluster through distributed shared memory and the
-// step's barrier spans the cluster.  A CTA (cluster) takes the heads blockIdx.x / kCluster, + stride, ...;
+// Every warp then sends its counts to all CTAs of the cluster through distributed shared memory.  A CTA (cluster) takes the heads blockIdx.x / kCluster, + stride, ...;
 // the scores of its next head stream into the staging area while it searches the current one.
 template <int kCluster>
 __global__ void __launch_bounds__(kThreads) select_sliced_kernel(ckv_shape s, int64_t unit_rows,
                                                                  const float* __restrict__ scores,
                                                                  const int32_t* __restrict__ budgets,
                                                                  const int32_t* __restrict__ offsets,
-                                                                 int32_t* __restrict__ indices) {
+                                                                 int32_t* __restrict__ indices, int* __restrict__ status) {
   extern __shared__ __align__(16) uint32_t stage[];   // [warps in use][1024] score bits in position order
-  __shared__ uint2 wcnt[2][kCluster][kWarps];
+  __shared__ __align__(8) uint2 wcnt[2][kCluster][kWarps];
   __shared__ uint32_t wtot[kWarps];
   __shared__ uint32_t ctot[kCluster];
+  __shared__ __align__(8) uint64_t xbar[2];   // one transaction barrier per buffer of wcnt
+  __shared__ volatile int dead_s;             // an exchange timed out here or in another CTA of the cluster
   pdl_launch_dependents();
+  if constexpr (kCluster > 1) {
+    if (threadIdx.x == 0) {
+      barrier_init(&xbar[0], 1), barrier_init(&xbar[1], 1);
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      dead_s = 0;
+    }
+    cooperative_groups::this_cluster().sync();   // nobody sends before every barrier of the cluster exists
+  }
+  uint32_t phase = 0;   // bit b: parity of the phase xbar[b] is in
   pdl_wait();   // budgets, offsets and scores come from the kernels before
   const int Hkv = s.n_kv_heads, W = s.window, n = s.seq_len - W;
   const int n_heads = s.n_units * Hkv, stride = (int)gridDim.x / kCluster;
@@ -88,9 +140,12 @@ __global__ void __launch_bounds__(kThreads) select_sliced_kernel(ckv_shape s, in
   const int wbase = warp * 1024;                            // first position of the warp inside the CTA
   const bool staged = cbase + wbase < n;                    // the warp holds positions of the prefix
   uint32_t* const ws = stage + wbase;
-  auto step_barrier = [&]() {
-    if constexpr (kCluster == 1) __syncthreads();
-    else cooperative_groups::this_cluster().sync();
+  // A CTA that gave up tells the others, and all CTAs of the cluster leave after the same cluster barrier:
+  // none sends to a CTA that is gone.
+  auto leave_dead = [&]() {
+    async_copy_wait();
+    if ((int)threadIdx.x < kCluster) *cooperative_groups::this_cluster().map_shared_rank(const_cast<int*>(&dead_s), threadIdx.x) = 1;
+    cooperative_groups::this_cluster().sync();
   };
   // every warp copies its own 1024 scores: nothing but the warp reads them
   auto prefetch = [&](int head) {
@@ -158,11 +213,24 @@ __global__ void __launch_bounds__(kThreads) select_sliced_kernel(ckv_shape s, in
       // the other buffer is written in the next step, this one again only after that step's barrier
       if constexpr (kCluster == 1) {
         if (lane == 0) wcnt[st & 1][0][warp] = make_uint2(r1, r2);
+        __syncthreads();
       } else {
+        uint64_t* bar = &xbar[st & 1];
+        if (threadIdx.x == 0) barrier_expect(bar, kCluster * kWarps * (int)sizeof(uint2));
         if (lane < kCluster)
-          *cooperative_groups::this_cluster().map_shared_rank(&wcnt[st & 1][rank][warp], lane) = make_uint2(r1, r2);
+          store_credit(cluster_address(&wcnt[st & 1][rank][warp], lane), (uint64_t)r1 | ((uint64_t)r2 << 32),
+                       cluster_address(bar, lane));
+        if (warp == 0 && !barrier_wait_bounded(bar, (phase >> (st & 1)) & 1u) && lane == 0) {
+          dead_s = 1;
+          atomicCAS(status, 0, kSelectTimeoutCode);
+        }
+        __syncthreads();   // warp 0 has seen every CTA's counts arrive
+        if (dead_s) {
+          leave_dead();
+          return;
+        }
+        phase ^= 1u << (st & 1);
       }
-      step_barrier();
       uint32_t wx = 0, wy = 0;   // lane l adds warp l of every CTA: both 16-bit fields stay below 2^14
 #pragma unroll
       for (int c = 0; c < kCluster; ++c) {
@@ -209,6 +277,10 @@ __global__ void __launch_bounds__(kThreads) select_sliced_kernel(ckv_shape s, in
       const uint32_t total = __reduce_add_sync(0xffffffffu, wt);
       if (warp == 0 && lane < kCluster) *cooperative_groups::this_cluster().map_shared_rank(&ctot[rank], lane) = total;
       cooperative_groups::this_cluster().sync();
+      if (dead_s) {   // set by a CTA that gave up, before this barrier
+        async_copy_wait();
+        return;
+      }
       for (int c = 0; c < rank; ++c) gt_before += (int)(ctot[c] & 0xffffu), eq_before += (int)(ctot[c] >> 16);
     }
     uint32_t m = gtp | eqp;
@@ -365,7 +437,7 @@ __global__ void __launch_bounds__(kThreads) select_digit_kernel(ckv_shape s, int
 
 template <int kCluster>
 cudaError_t launch_sliced(const ckv_shape& s, int n, int64_t unit_rows, const float* scores, const int32_t* budgets,
-                          const int32_t* offsets, int32_t* indices, cudaStream_t st) {
+                          const int32_t* offsets, int32_t* indices, int* status, cudaStream_t st) {
   const int per_cta = (n + kCluster - 1) / kCluster;   // staging covers the fullest CTA
   const size_t smem = (size_t)((std::min(per_cta, kSlicedMax) + 1023) / 1024) * 1024 * sizeof(uint32_t);
   cudaError_t e = cudaFuncSetAttribute(select_sliced_kernel<kCluster>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -399,21 +471,21 @@ cudaError_t launch_sliced(const ckv_shape& s, int n, int64_t unit_rows, const fl
   }
   const int n_heads = s.n_units * s.n_kv_heads;
   cfg.gridDim = dim3((unsigned)(std::min(n_heads, resident) * kCluster));
-  return cudaLaunchKernelEx(&cfg, select_sliced_kernel<kCluster>, s, unit_rows, scores, budgets, offsets, indices);
+  return cudaLaunchKernelEx(&cfg, select_sliced_kernel<kCluster>, s, unit_rows, scores, budgets, offsets, indices, status);
 }
 
 }  // namespace
 
 cudaError_t launch_select(const ckv_shape& s, const ckv_params& p, const float* scores, const int32_t* budgets,
-                          const int32_t* offsets, int32_t* indices, cudaStream_t st) {
+                          const int32_t* offsets, int32_t* indices, int* status, cudaStream_t st) {
   const int n = s.seq_len - s.window;
   // unit u's indices start at u * unit_rows; its heads' budgets fill that exactly unless the selection is elastic
   const int64_t unit_rows = (int64_t)s.n_kv_heads * (p.budget_per_head < s.seq_len ? p.budget_per_head : s.seq_len);
   cudaError_t e;
-  if (n <= kSlicedMax) e = launch_sliced<1>(s, n, unit_rows, scores, budgets, offsets, indices, st);
-  else if (n <= 2 * kSlicedMax) e = launch_sliced<2>(s, n, unit_rows, scores, budgets, offsets, indices, st);
-  else if (n <= 4 * kSlicedMax) e = launch_sliced<4>(s, n, unit_rows, scores, budgets, offsets, indices, st);
-  else if (n <= 8 * kSlicedMax) e = launch_sliced<8>(s, n, unit_rows, scores, budgets, offsets, indices, st);
+  if (n <= kSlicedMax) e = launch_sliced<1>(s, n, unit_rows, scores, budgets, offsets, indices, status, st);
+  else if (n <= 2 * kSlicedMax) e = launch_sliced<2>(s, n, unit_rows, scores, budgets, offsets, indices, status, st);
+  else if (n <= 4 * kSlicedMax) e = launch_sliced<4>(s, n, unit_rows, scores, budgets, offsets, indices, status, st);
+  else if (n <= 8 * kSlicedMax) e = launch_sliced<8>(s, n, unit_rows, scores, budgets, offsets, indices, status, st);
   else {
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(s.n_units * s.n_kv_heads), cfg.blockDim = dim3(kThreads), cfg.stream = st;
