@@ -114,7 +114,7 @@ struct __align__(16) Desc {
   int first;      // P1: this group's first tile of the run (reset the running pair)
                   // P2: index (u * Hkv + g) of the KV group
   int head0;      // P2: index (u * H + head) of the first query head of the row block
-  int n_heads;    // P2: query heads of the row block that exist
+  int n_heads;    // query heads of the row block that exist
   int nbias_buf;  // P2: which bias vector belongs to the tile's chunk
 };
 
@@ -476,7 +476,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         if (ln.type == kP1) {
           d[0] = make_int4(ln.type | (q_phase << 9), ln.chunk, tile,
                            (ln.k + 2 >= ln.tr) ? ln.ric * a.ppr + (ln.k & 1) : -1);
-          d[1] = make_int4(ln.k < 2, 0, 0, 0);
+          d[1] = make_int4(ln.k < 2, 0, ln.heads, 0);
         } else {
           d[0] = make_int4(ln.type | (q_phase << 9), ln.chunk, tile, ln.u * (int)a.hw_stride + ln.head0);
           d[1] = make_int4(ln.u * a.Hkv + ln.g, ln.u * a.H + ln.head0, ln.heads, ln.gen % kBiasBufs);
@@ -688,6 +688,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         // ---------------------------------------------------------- P1: running (max, sum) of this row
         if (d.first) m_run = kMinRowMax, l_run = 0.f;
         const int limit = a.n + row % W;   // last key this window row sees
+        if (!kGrouped && quad * 32 >= d.n_heads * W) {
+          // a short row block (the group's last heads): none of this warp's rows exists, nothing reads their pair
+          // (the grouped output is only chosen when the heads fill the block)
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_empty);
+        } else {
 #pragma unroll 1
         for (int cc = 0; cc < 4; ++cc) {
           float v[32];
@@ -731,6 +737,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
             part = slice_sum(m_run);
           }
           l_run += part;
+        }
         }
         if (d.part_slot >= 0) {
           // this group's last tile of the run: publish the pair; the last warp of the chunk's
@@ -783,8 +790,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
             msum += c;
           }
         };
+        // a short row block has fewer slices of query rows (never with the grouped output)
+        const int cc_end = kGrouped ? 4 : min(4, (d.n_heads * W + 31) / 32);
 #pragma unroll 1
-        for (int cc = 0; cc < 4; ++cc) {
+        for (int cc = 0; cc < cc_end; ++cc) {
           float v[32];
           tmem_ld32(taddr + cc * 32, v);
           uint64_t acc2[kHeadsPerSlice];   // per head of the slice: two running sums
@@ -817,7 +826,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           float acc[kHeadsPerSlice][2];
 #pragma unroll
           for (int hh = 0; hh < kHeadsPerSlice; ++hh) unpack2(acc2[hh], acc[hh][0], acc[hh][1]);
-          if (cc == 3) {  // all bias reads and TMEM loads of this sub-item are done
+          if (cc == cc_end - 1) {  // all bias reads and TMEM loads of this sub-item are done
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_empty);
