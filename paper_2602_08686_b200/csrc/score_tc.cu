@@ -574,15 +574,17 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       bool staged = false;
       if (ready_mask & 1u) {
         // nbias[G % kBiasBufs] last served run G - kBiasBufs: all of its tiles must have been issued, and a
-        // tile's readers are done once the producer has got kStages + kTmemBufs sub-items past it (it waits
-        // for the K stage of sub-item j - kStages to be free, whose MMA waited for the TMEM buffer of
-        // sub-item j - kStages - kTmemBufs).
+        // tile's readers are done once the producer has got kStages + 2 kTmemBufs sub-items past it (it waits
+        // for the K stage of sub-item j - kStages to be free, whose MMA waited for the release of the TMEM
+        // buffer by sub-item j - kStages - kTmemBufs; a warp releases a sub-item's buffer after its last
+        // accumulator load and before that slice's math, so what is certain then is that it has finished
+        // all math, bias reads included, of its sub-item before, j - kStages - 2 kTmemBufs).
         bool free_buf = true;
         if (G > kBiasBufs) {
           free_buf = *(volatile int*)&sm.gen_fin[G % kBiasBufs] == G - kBiasBufs;
           if (free_buf) {
             __threadfence_block();
-            free_buf = *(volatile int*)&sm.prod_j >= *(volatile int*)&sm.gen_last_j[G % kBiasBufs] + kStages + kTmemBufs;
+            free_buf = *(volatile int*)&sm.prod_j >= *(volatile int*)&sm.gen_last_j[G % kBiasBufs] + kStages + 2 * kTmemBufs;
           }
         }
         free_buf = __shfl_sync(0xffffffffu, free_buf ? 1 : 0, 0) != 0;
@@ -796,6 +798,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         for (int cc = 0; cc < cc_end; ++cc) {
           float v[32];
           tmem_ld32(taddr + cc * 32, v);
+          if (cc == cc_end - 1) {  // all TMEM loads of this sub-item are done: the next tile's MMAs may run during the math
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_empty);
+          }
           uint64_t acc2[kHeadsPerSlice];   // per head of the slice: two running sums
 #pragma unroll
           for (int hh = 0; hh < kHeadsPerSlice; ++hh) acc2[hh] = pack2(0.f, 0.f);
@@ -826,11 +833,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           float acc[kHeadsPerSlice][2];
 #pragma unroll
           for (int hh = 0; hh < kHeadsPerSlice; ++hh) unpack2(acc2[hh], acc[hh][0], acc[hh][1]);
-          if (cc == cc_end - 1) {  // all bias reads and TMEM loads of this sub-item are done
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_empty);
-          }
           if (W >= 32) {
             head_acc += acc[0][0] + acc[0][1];
             const int rows_done = (cc + 1) * 32;
