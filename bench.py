@@ -34,8 +34,8 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of score_tc_kernel per unit, from an ncu capture of an 8-unit
 # launch of the workload's shape (profiles/score_tc_kernel_c2_8units.md; 2 units for the 128k shape); a launch's traffic is this times its
 # units (every unit streams its own K once per pass).  Workloads without a capture of the current kernel: none.
-SCAN_DRAM_TRAFFIC_PER_UNIT = {"c2": (1.019774e9 + 7.897344e6) / 8, "c3": (1.019774e9 + 7.897344e6) / 8,
-                              "c4": (1.014323456e9 + 6.933248e6) / 2}
+SCAN_DRAM_TRAFFIC_PER_UNIT = {"c2": (1.020698e9 + 8.101632e6) / 8, "c3": (1.020698e9 + 8.101632e6) / 8,
+                              "c4": (1.014879488e9 + 7.535616e6) / 2}
 
 
 def measured_peaks():
