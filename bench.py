@@ -68,6 +68,11 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.rows.append((time.time(), line.strip()))
 
+    def wait_first_row(self, limit_s: float) -> None:
+        t_end = time.time() + limit_s
+        while self.proc is not None and not self.rows and time.time() < t_end:
+            time.sleep(0.01)
+
     def stop(self, t0: float, t1: float) -> dict:
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
@@ -223,10 +228,13 @@ def main():
     scan_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     for a_, b_ in scan_ev:       # a first record creates the handles
         a_.record(), b_.record()
+    # the clock sampler runs from before the warm-up (nvidia-smi takes a while to print its first row on a fresh box)
+    sampler = ClockSampler(local_rank) if rank == 0 else None
     for _ in range(max(args.warmup, 3)):
         step()
+    if sampler is not None:
+        sampler.wait_first_row(3.0)
     barrier()
-    sampler = ClockSampler(local_rank) if rank == 0 else None
     launches0 = B.ckv_kernel_launches()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0 = time.time()
