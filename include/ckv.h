@@ -19,7 +19,7 @@
  *   - Errors are return codes.  Argument errors are found on the host before
  *     anything is launched (CKV_ERR_INVALID_ARG / UNSUPPORTED / WORKSPACE); a CUDA
  *     launch error gives CKV_ERR_CUDA.  A device-side wait that ran out of its
- *     iteration limit is recorded in the work space's status word and read back
+ *     time limit (2 s) is recorded in the work space's status word and read back
  *     with ckv_device_status().
  *   - Preconditions that are not checked: inputs are finite, head_w >= 0.
  *   - Layouts: q_win [Nu, H, W, d], k and v [Nu, Hkv, L, d]; the last dimension is
@@ -196,7 +196,8 @@ ckv_status ckv_unit_max(const ckv_shape* shape, const ckv_params* params, float*
  * largest of scores[g,0:n] are kept, equal scores resolved toward the lowest index; the kept
  * positions are written in ascending order and followed by the window n .. L-1, which is always
  * retained.  indices [Nu, Hkv * min(B,L)] int32, head g of unit u at row offsets[u,g] of the unit's
- * Hkv * min(B,L) rows.
+ * Hkv * min(B,L) rows.  Of the work space only the status word is used: prefixes longer than 32768
+ * are searched by clusters of CTAs, whose bounded exchange wait reports there (ckv_device_status).
  */
 ckv_status ckv_select(const ckv_shape* shape, const ckv_params* params, const float* scores,
                       const int32_t* budgets, const int32_t* offsets, int32_t* indices, void* ws,
