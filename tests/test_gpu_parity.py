@@ -468,6 +468,37 @@ def test_select_distributions(B, n, dist):
     np.testing.assert_array_equal(idx.cpu().numpy(), want)
 
 
+@pytest.mark.parametrize("n,Nu", [(20000, 80), (40000, 48), (140000, 24)])
+def test_select_many_heads_per_cta(B, n, Nu):
+    """More heads than the device holds CTAs (clusters of 1, 2 and 8): every CTA loops over several heads, with the
+    next head's scores streaming in during the search, and heads that keep nothing or everything of the prefix
+    sit between heads that are searched."""
+    Hkv, W = 4, 32
+    L = n + W
+    rng = np.random.default_rng(n + Nu)
+    scores = rng.lognormal(0.0, 2.0, (Nu, Hkv, n)).astype(np.float32)
+    scores[:, :, ::7] = np.float32(1.5)          # many equal scores, some of them at the cut
+    a, b = 480, n // 5
+    b += (-(a + b + n)) % 4
+    kinds = np.array([0, n, a, b], np.int32)     # nothing, everything, few, many
+    budgets = np.stack([np.roll(kinds, u % 4) for u in range(Nu)]) + W
+    rows = int(budgets[0].sum())
+    assert rows % Hkv == 0
+    offsets = np.concatenate([np.zeros((Nu, 1), np.int32), budgets.cumsum(1).astype(np.int32)], 1)
+    q = torch.zeros(Nu, Hkv, W, 128, dtype=torch.bfloat16, device="cuda")
+    k = torch.zeros(Nu, Hkv, L, 128, dtype=torch.bfloat16, device="cuda")   # only its shape is used
+    shape = B.make_shape(q, k)
+    params = B.make_params(B.Params(budget_per_head=rows // Hkv, floor_per_head=0), None, None)
+    ws = B.alloc_workspace(shape, params, "cuda")
+    idx = torch.full((Nu, rows), -1, dtype=torch.int32, device="cuda")
+    B.ckv_select(shape, params, torch.from_numpy(scores).cuda(), torch.from_numpy(budgets).cuda(),
+                 torch.from_numpy(offsets).cuda(), idx, ws)
+    assert B.ckv_device_status(ws) == B.OK
+    prob = Problem(Nu, Hkv, Hkv, L, W, budget_per_head=rows // Hkv)
+    want = oracle.select(prob, scores.astype(np.float64), budgets, offsets)
+    np.testing.assert_array_equal(idx.cpu().numpy(), want)
+
+
 def test_strided_inputs(B):
     """K/V living inside a larger allocation (non-dense unit/head/token strides) give the same result."""
     cfg = gen.shrink(gen.CONFIGS["c2"], n_layers=2, n_q_heads=8, n_kv_heads=2, seq_len=700, budget_per_head=64,
