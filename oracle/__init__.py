@@ -41,7 +41,8 @@ class _Params(C.Structure):
                 ("pool_kind", "pool_size", "budget_per_head", "floor_per_head", "n_buckets",
                  "bucket_override", "head_w_per_unit", "sens_per_unit", "value_norm")] + \
                [("value_norm_eps", C.c_float), ("shared_elastic", C.c_int32), ("global_alpha", C.c_int32),
-                ("units_per_prompt", C.c_int32)]
+                ("units_per_prompt", C.c_int32), ("gate_layers", C.c_int32), ("ppl_bins", C.c_int32),
+                ("budget_levels", C.c_int32), ("gate_coords", C.c_void_p)]
 
 
 @dataclass
@@ -67,6 +68,13 @@ class Problem:
     shared_elastic: bool = False      # the paper's own selection: one elastic set per unit (Eq. 6 over all heads, Eq. 8)
     global_alpha: bool = False        # Alg. 1 (A): alpha and the risk coordinate from the mean over the prompt's layers and heads
     units_per_prompt: int = 1         # layers per prompt (consecutive units) for global_alpha
+    # The gate table as the paper indexes it (Sec. 4.3, Alg. 1 (D)): with gate_layers > 0 the table passed as `sens`
+    # is [gate_layers, n_buckets, ppl_bins, budget_levels] and gate_coords [Nu,3] int32 gives each unit's
+    # (layer row, perplexity bin, budget level).
+    gate_layers: int = 0
+    ppl_bins: int = 1
+    budget_levels: int = 1
+    gate_coords: object = None
 
     @property
     def n(self) -> int:
@@ -81,10 +89,16 @@ class Problem:
                       self.window, self.dtype)
 
     def _params(self) -> _Params:
+        coords = None
+        if self.gate_layers > 0:
+            # kept on the object so that the array outlives the C call
+            self._coords = np.ascontiguousarray(self.gate_coords, np.int32).reshape(self.n_units, 3)
+            coords = self._coords.ctypes.data_as(C.c_void_p)
         return _Params(self.pool_kind, self.pool_size, self.budget_per_head, self.floor_per_head,
                        self.n_buckets, self.bucket_override, int(self.head_w_per_unit),
                        int(self.sens_per_unit), int(self.value_norm), float(self.value_norm_eps),
-                       int(self.shared_elastic), int(self.global_alpha), int(self.units_per_prompt))
+                       int(self.shared_elastic), int(self.global_alpha), int(self.units_per_prompt),
+                       int(self.gate_layers), int(self.ppl_bins), int(self.budget_levels), coords)
 
 
 _lib = None
@@ -270,6 +284,16 @@ def attend(prob: Problem, q_dec, k, v, budgets=None, offsets=None):
                                _p(budgets), _p(offsets), C.c_int64(k.shape[1] if compressed else 0), _p(out), _p(lse)),
            "attend")
     return out, lse
+
+
+def depth_map(table, n_dst: int) -> np.ndarray:
+    """A table [n_src, ...] compiled for n_src layers, mapped to n_dst layers by relative depth (fp32)."""
+    src = np.ascontiguousarray(table, np.float32)
+    n_src = src.shape[0]
+    row = int(np.prod(src.shape[1:])) if src.ndim > 1 else 1
+    dst = np.empty((n_dst,) + src.shape[1:], np.float32)
+    _check(lib().oracle_depth_map(_p(src), C.c_int(n_src), C.c_int(n_dst), C.c_int64(row), _p(dst)), "depth_map")
+    return dst
 
 
 def num_threads() -> int:

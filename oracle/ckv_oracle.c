@@ -22,7 +22,9 @@
  *       u_h[t] = pooled_h[t] * rho_g[t]                    (Eq. 4, Alg. 1 (B))
  *   O6  head table u_g[t] = max_{h in group g} W_head[h] * u_h[t]       (Eq. 6)
  *   O7  risk coordinate: entropy of the normalised window mass, bucket,
- *       threshold tau = table[bucket]                    (Eq. 7 left, Alg. 1 (A),(D))
+ *       threshold tau = table[bucket]                    (Eq. 7 left, Alg. 1 (A),(D));
+ *       with gate_layers set the table is the paper's T_gate[l, b_ent, b_ppl, B_l]
+ *       (Sec. 4.3), the perplexity bin and the layer / budget rows supplied per unit
  *   O8  candidate counts under tau (Eq. 8's candidate set) -> per-head budgets
  *       clamped so that they sum to the total budget
  *   O9  Top-k per KV head, ties to the lowest index, window always kept (Eq. 8)
@@ -40,7 +42,8 @@
  * one-hot distributions, hand-computed norms, the mean identity and scale
  * invariance of O5b, brute-force rational water-filling for O8, brute-force
  * sorting for O9, direct indexing for O10, FullKV reproduction, and the
- * identity |p - p~|_1 = 2m of Eq. A2.
+ * identity |p - p~|_1 = 2m of Eq. A2, a hand-built gate table with one distinct
+ * value per cell, and numpy's linear interpolation for the depth mapping.
  * Parity unpinned by the paper itself (the paper has no such step; pinned only
  * by the invariants above): the O8 redistribution rule, the bucket edges of O7,
  * and the edge rule of the O5 pooling.
@@ -77,6 +80,12 @@ typedef struct {
   int32_t shared_elastic;  /* 1: one elastic set per unit (Eq. 6 over all heads, Eq. 8), shared by its KV heads */
   int32_t global_alpha;    /* 1: alpha from the mean attention over all layers and heads of the prompt */
   int32_t units_per_prompt; /* layers of one prompt: units [s N, (s + 1) N) belong to prompt s (global_alpha) */
+  /* The threshold table as the paper indexes it (Sec. 4.3, Alg. 1 (D)): tau = T_gate[l, b_ent, b_ppl, B_l].
+   * gate_layers > 0 switches it on: the table argument is then [gate_layers][n_buckets][ppl_bins][budget_levels]
+   * (n_buckets entropy bins) and gate_coords [Nu,3] holds, per unit, the layer row l, the perplexity bin b_ppl
+   * (computed by the caller from the language model's logits, Eq. 7 right) and the index of the budget level. */
+  int32_t gate_layers, ppl_bins, budget_levels;
+  const int32_t *gate_coords;
 } or_params;
 
 /* exact widening of an input element to double */
@@ -369,15 +378,23 @@ int oracle_allocate(int Hkv, int64_t n, int64_t f, int64_t P, const int64_t *dem
         given += e[g];
       }
     }
+    /* hand the left-over rows out: the free heads in the order (larger fractional part first, lower head index
+       first among equal parts) each take one row until none is left */
     int64_t left = (D > 0) ? R - given : 0;
-    while (left > 0) {
-      int best = -1;
-      for (int g = 0; g < Hkv; ++g)
-        if (rem[g] > 0 && (best < 0 || rem[g] > rem[best])) best = g;
-      if (best < 0) return 3; /* cannot happen: left < number of non-zero remainders */
-      e[best] += 1;
-      rem[best] = -1;
-      --left;
+    int order[64], n_free = 0;
+    for (int g = 0; g < Hkv; ++g) {
+      if (rem[g] < 0) continue;
+      int at = n_free++;
+      while (at > 0 && rem[order[at - 1]] < rem[g]) { /* strictly smaller parts move back: equal parts keep head order */
+        order[at] = order[at - 1];
+        --at;
+      }
+      order[at] = g;
+    }
+    if (left > n_free) return 3; /* cannot happen: the fractional parts sum to `left` and each is below one */
+    for (int r = 0; r < left; ++r) {
+      if (rem[order[r]] == 0) return 3;
+      e[order[r]] += 1;
     }
     return 0;
   }
@@ -397,7 +414,16 @@ int oracle_budget(const or_shape *s, const or_params *p, const double *scores, c
     int b;
     risk_bucket(colmass + (int64_t)u * L, L, W, H, p->n_buckets, &ent, &b);
     if (p->bucket_override >= 0) b = p->bucket_override < p->n_buckets ? p->bucket_override : p->n_buckets - 1;
-    const double tau = (double)sens[(p->sens_per_unit ? (int64_t)u * p->n_buckets : 0) + b];
+    double tau;
+    if (p->gate_layers > 0) { /* Alg. 1 (D): tau = T_gate[l, b_ent, b_ppl, B_l], row-major */
+      if (!p->gate_coords || p->ppl_bins < 1 || p->budget_levels < 1) return 1;
+      const int32_t *c = p->gate_coords + (int64_t)u * 3;
+      const int l = c[0], bp = c[1], bb = c[2];
+      if (l < 0 || l >= p->gate_layers || bp < 0 || bp >= p->ppl_bins || bb < 0 || bb >= p->budget_levels) return 1;
+      tau = (double)sens[(((int64_t)l * p->n_buckets + b) * p->ppl_bins + bp) * p->budget_levels + bb];
+    } else {
+      tau = (double)sens[(p->sens_per_unit ? (int64_t)u * p->n_buckets : 0) + b];
+    }
     bucket[u] = b;
     entropy[u] = ent;
     if (tau_out) tau_out[u] = tau;
@@ -592,6 +618,26 @@ int oracle_kept_mass(const or_shape *s, const void *q, const void *k, const int3
       }
       free(row);
     }
+  return 0;
+}
+
+/* ------------------------------------------------------------------ depth mapping of a compiled table
+ * A table compiled for n_src layers is reused on a model of n_dst layers by relative depth (the appendix on
+ * cross-architecture use: "monotonic depth mapping, e.g. relative-depth interpolation"): target layer l sits
+ * at relative depth r = l / (n_dst - 1), i.e. at position x = r (n_src - 1) of the source's layer axis, and
+ * takes the linear interpolation of the two source rows around x.  First and last layers map onto first and
+ * last; n_dst == n_src is the identity.  src [n_src,row], dst [n_dst,row], fp32 tables, arithmetic in double. */
+int oracle_depth_map(const float *src, int n_src, int n_dst, int64_t row, float *dst) {
+  if (n_src < 1 || n_dst < 1 || row < 1) return 1;
+  for (int l = 0; l < n_dst; ++l) {
+    const double x = (n_dst > 1) ? (double)l * (double)(n_src - 1) / (double)(n_dst - 1) : 0.0;
+    int lo = (int)floor(x);
+    if (lo > n_src - 1) lo = n_src - 1;
+    const int hi = lo + 1 < n_src ? lo + 1 : n_src - 1;
+    const double w = x - (double)lo;
+    for (int64_t c = 0; c < row; ++c)
+      dst[(int64_t)l * row + c] = (float)((1.0 - w) * (double)src[(int64_t)lo * row + c] + w * (double)src[(int64_t)hi * row + c]);
+  }
   return 0;
 }
 

@@ -243,6 +243,83 @@ def test_allocate_matches_rational_brute_force():
     assert cases == 1600
 
 
+def iterative_allocate(n, f, P, dem):
+    """The budget clamp stated as a fixed-point loop (reading of the clamp-to-total rule): share the rows in
+    proportion to the demands; pin every head whose share falls below the floor at the floor and take it out;
+    when no head is below the floor, pin every head whose share exceeds the cap at the cap; repeat until nothing
+    is pinned.  Exact integer comparisons; then floor plus largest remainders, ties to the lowest head."""
+    dem = [int(x) for x in dem]
+    active = list(range(len(dem)))
+    e = [None] * len(dem)
+    R = P
+    while active:
+        D = sum(dem[g] for g in active)
+        low = [g for g in active if R * dem[g] < f * D]
+        if low:
+            for g in low:
+                e[g] = f
+            R -= f * len(low)
+            active = [g for g in active if g not in low]
+            continue
+        high = [g for g in active if R * dem[g] > n * D]
+        if high:
+            for g in high:
+                e[g] = n
+            R -= n * len(high)
+            active = [g for g in active if g not in high]
+            continue
+        break
+    if active:
+        D = sum(dem[g] for g in active)
+        for g in active:
+            e[g] = R * dem[g] // D
+        left = R - sum(e[g] for g in active)
+        for g in sorted(active, key=lambda g: (-((R * dem[g]) % D), g))[:left]:
+            e[g] += 1
+    return e
+
+
+def test_allocate_matches_the_iterative_statement_at_workload_sizes():
+    """Eight KV heads and prefixes up to 131040 (the workloads' sizes), where the rational brute force is too slow:
+    the water-filling oracle against the fixed-point loop, an independent statement of the same rule."""
+    rng = np.random.default_rng(5)
+    cases = 0
+    for Hkv, n, W in ((8, 32736, 32), (8, 131040, 32), (4, 65472, 64), (8, 2016, 32), (2, 2016, 32)):
+        for _ in range(600):
+            B = int(rng.choice([128, 512, 2048, int(rng.integers(W + 1, n))]))
+            B = max(W + 1, min(B, n))
+            f = int(rng.choice([0, 1, 8, int(rng.integers(0, B - W + 1))]))
+            f = min(f, B - W)
+            P = Hkv * (B - W)
+            style = rng.integers(0, 4)
+            if style == 0:      # counts of scores above a threshold: anywhere in [0, n]
+                dem = rng.integers(0, n + 1, Hkv)
+            elif style == 1:    # a few starved heads next to saturated ones
+                dem = np.where(rng.random(Hkv) < 0.4, rng.integers(0, 4, Hkv), rng.integers(n // 2, n + 1, Hkv))
+            elif style == 2:    # near-equal demands: the remainders decide
+                dem = int(rng.integers(1, n)) + rng.integers(0, 3, Hkv)
+            else:               # small demands: many heads at the floor or at the cap
+                dem = rng.integers(0, 2 * (B - W) + 2, Hkv)
+            dem = np.clip(dem, max(f, 1), n)
+            got = list(oracle.allocate(n, f, P, dem))
+            assert got == iterative_allocate(n, f, P, dem), (Hkv, n, f, P, dem)
+            assert sum(got) == P and min(got) >= f and max(got) <= n
+            cases += 1
+    assert cases == 3000
+
+
+def test_allocate_iterative_statement_agrees_with_rational_brute_force():
+    """The two pins against each other on small cases (so that neither is only checked through the oracle)."""
+    rng = np.random.default_rng(6)
+    for _ in range(500):
+        Hkv = int(rng.integers(1, 6))
+        n = int(rng.integers(1, 40))
+        f = int(rng.integers(0, n + 1))
+        P = int(rng.integers(f * Hkv, n * Hkv + 1))
+        dem = rng.integers(max(f, 1), max(f, 1, n) + 1, Hkv)
+        assert iterative_allocate(n, f, P, dem) == brute_allocate(n, f, P, dem), (n, f, P, dem)
+
+
 def test_allocate_two_sided_clamp_case():
     """A tiny demand next to a huge one: the low head sits at the floor, the high head at the cap."""
     assert list(oracle.allocate(10, 2, 18, [1, 1000])) == [8, 10]
@@ -634,3 +711,83 @@ def test_attend_against_library_softmax_and_the_discarded_mass_identity(dtype):
     out_f, lse_f = oracle.attend(prob, gen.as_numpy(qd), full["k_out"], full["v_out"], full["budgets"], full["offsets"])
     np.testing.assert_allclose(out_f, out, rtol=1e-12, atol=1e-14)
     np.testing.assert_allclose(lse_f, lse, rtol=1e-13)
+
+
+# ----------------------------------------------------------------------------- the gate table (Sec. 4.3, Alg. 1 (D))
+def test_gate_table_lookup_reaches_every_cell():
+    """tau = T_gate[l, b_ent, b_ppl, B_l] (Alg. 1 (D)) on the paper's 20 x 4 entropy x perplexity grid: a hand-built
+    table with a different value in every cell; the entropy bin is forced through bucket_override and the other
+    coordinates come per unit, so every cell of the grid is reached and must come back as the threshold."""
+    n_layers, n_ent, n_ppl, n_bud = 3, 20, 4, 2
+    cells = n_layers * n_ent * n_ppl * n_bud
+    table = (0.8 + 0.2 * np.random.default_rng(3).permutation(cells) / cells).astype(np.float32)
+    table = table.reshape(n_layers, n_ent, n_ppl, n_bud)
+    assert len(set(table.ravel().tolist())) == cells
+    prob, q, k, _ = rand_case(21, Nu=n_layers * n_bud, H=4, Hkv=2, L=64, W=8)
+    s, cm = oracle.score(prob, gen.as_numpy(q), gen.as_numpy(k), np.ones((prob.n_units, 4), np.float32))
+    prob.n_buckets, prob.gate_layers, prob.ppl_bins, prob.budget_levels = n_ent, n_layers, n_ppl, n_bud
+    seen = set()
+    for b_ent in range(n_ent):
+        for b_ppl in range(n_ppl):
+            coords = [(u // n_bud, b_ppl, u % n_bud) for u in range(prob.n_units)]
+            prob.gate_coords, prob.bucket_override = coords, b_ent
+            out = oracle.budget(prob, s, cm, table)
+            for u, (l, p, b) in enumerate(coords):
+                assert out["tau"][u] == table[l, b_ent, p, b]
+                # and the threshold is the one the counts were taken with
+                assert (out["counts"][u] == (s[u] >= float(table[l, b_ent, p, b])).sum(-1)).all()
+                seen.add((l, b_ent, p, b))
+    assert len(seen) == cells
+
+
+def test_gate_table_takes_its_entropy_bin_from_the_window_mass():
+    """Without an override the first table axis is the entropy bin of Eq. 7: uniform mass gives the last of the
+    20 bins, mass on one position the first."""
+    L, W, H = 50, 4, 2
+    prob = Problem(1, H, 1, L, W, head_dim=16, dtype=oracle.F32, budget_per_head=20, n_buckets=20,
+                   gate_layers=1, ppl_bins=4, budget_levels=1, gate_coords=[(0, 2, 0)])
+    table = np.arange(80, dtype=np.float32).reshape(1, 20, 4, 1)
+    scores = np.zeros((1, 1, L - W))
+    uniform = np.full((1, L), W * H / L)
+    assert oracle.budget(prob, scores, uniform, table)["tau"][0] == table[0, 19, 2, 0]
+    one_hot = np.zeros((1, L))
+    one_hot[0, 7] = W * H
+    assert oracle.budget(prob, scores, one_hot, table)["tau"][0] == table[0, 0, 2, 0]
+
+
+def test_gate_coordinates_out_of_range_are_refused():
+    prob, q, k, _ = rand_case(22, Nu=1)
+    s, cm = oracle.score(prob, gen.as_numpy(q), gen.as_numpy(k), np.ones((1, 4), np.float32))
+    prob.gate_layers, prob.ppl_bins, prob.budget_levels = 2, 4, 1
+    table = np.ones((2, prob.n_buckets, 4, 1), np.float32)
+    for bad in [(2, 0, 0), (0, 4, 0), (0, 0, 1), (-1, 0, 0)]:
+        prob.gate_coords = [bad]
+        with pytest.raises(RuntimeError):
+            oracle.budget(prob, s, cm, table)
+
+
+@pytest.mark.parametrize("n_src,n_dst", [(32, 32), (32, 28), (32, 40), (32, 80), (2, 7), (5, 1), (1, 6)])
+def test_depth_map_is_relative_depth_interpolation(n_src, n_dst):
+    """Reuse of a table compiled for one depth on a model of another (the appendix on cross-architecture use):
+    numpy's piecewise-linear interpolation over relative depth is the same map; same depth is the identity, first
+    and last layers map onto first and last, and a table that rises with depth still rises."""
+    rng = np.random.default_rng(n_src * 100 + n_dst)
+    src = rng.uniform(0.8, 1.0, (n_src, 20, 4)).astype(np.float32)
+    got = oracle.depth_map(src, n_dst)
+    assert got.shape == (n_dst, 20, 4) and got.dtype == np.float32
+    xs = np.linspace(0.0, 1.0, n_src) if n_src > 1 else np.zeros(1)
+    xd = np.linspace(0.0, 1.0, n_dst) if n_dst > 1 else np.zeros(1)
+    want = np.stack([np.interp(xd, xs, src[:, i, j].astype(np.float64)) for i in range(20) for j in range(4)], -1)
+    np.testing.assert_allclose(got.reshape(n_dst, 80), want, rtol=1e-6, atol=0)
+    if n_dst == n_src:
+        np.testing.assert_array_equal(got, src)
+    np.testing.assert_array_equal(got[0], src[0])
+    if n_dst > 1:
+        np.testing.assert_array_equal(got[-1], src[-1])
+    rising = np.sort(src, axis=0)
+    assert (np.diff(oracle.depth_map(rising, n_dst).astype(np.float64), axis=0) >= 0).all()
+    # a table that is linear in depth stays linear in relative depth (closed form)
+    lin = (0.8 + 0.2 * np.arange(n_src) / max(n_src - 1, 1)).astype(np.float32).reshape(n_src, 1)
+    if n_src > 1 and n_dst > 1:
+        np.testing.assert_allclose(oracle.depth_map(lin, n_dst)[:, 0], 0.8 + 0.2 * np.arange(n_dst) / (n_dst - 1),
+                                   rtol=1e-6)
