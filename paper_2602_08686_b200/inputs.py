@@ -117,10 +117,20 @@ def make_unit(cfg: Config, unit: int, device="cpu"):
     qbar = qf.mean(1)
     k[:, 0, :] = 4.0 * math.sqrt(d) * qbar / qbar.norm(dim=-1, keepdim=True)
 
-    # needles: cosine 0.9 to one window query of the group, norm sqrt(d)
+    # needles: cosine 0.9 to one window query of the group, norm sqrt(d).  The query is drawn from the half of the
+    # group's rows that point least along the sink direction (a row that points along it hands the sink nearly all
+    # of its attention, and a key planted for that row would not stand out), each row at most once where the group
+    # has enough of them, so that two needles never split one row's attention.
     pos = _needle_positions(cfg, gen, dev)
     nn = cfg.n_needles
-    pick = torch.randint(0, G * W, (Hkv, nn), generator=gen, device=dev)
+    along = (qf * (qbar / qbar.norm(dim=-1, keepdim=True)).unsqueeze(1)).sum(-1)
+    eligible = along.argsort(dim=1)[:, :(G * W + 1) // 2]
+    m = eligible.shape[1]
+    if nn <= m:
+        sel = torch.rand(Hkv, m, generator=gen, device=dev).argsort(dim=1)[:, :nn]
+    else:
+        sel = torch.randint(0, m, (Hkv, nn), generator=gen, device=dev)
+    pick = torch.gather(eligible, 1, sel)
     qsel = torch.gather(qf, 1, pick.unsqueeze(-1).expand(Hkv, nn, d))
     qhat = qsel / qsel.norm(dim=-1, keepdim=True)
     z = torch.randn(Hkv, nn, d, generator=gen, device=dev)

@@ -43,6 +43,15 @@ def needle_census(cfg, b, idx, bud, off):
     return planted, kept, lost
 
 
+def dropped_needles(cfg, needles, idx_u, off_u):
+    """{(head, position)} of the planted needles that one unit's selection leaves out."""
+    out = set()
+    for g in range(cfg.n_kv_heads):
+        s = set(idx_u[off_u[g]:off_u[g + 1]].tolist())
+        out |= {(g, int(t)) for t in needles[g].tolist() if int(t) not in s}
+    return out
+
+
 def run_full(B, cfg, units, sample, census=True):
     """One fused call over `units`; oracle comparison on the positions `sample` of that list."""
     b = gen.make_batch(cfg, "cuda", units)
@@ -79,13 +88,23 @@ def run_full(B, cfg, units, sample, census=True):
         # and against the oracle's own scores: differences only inside the near-tie band
         ref["scores"], ref["idx"] = sc, oracle.select(prob1, sc, ref["budgets"], ref["offsets"])
         check_selection_against_oracle(idx[j:j + 1], bud[j:j + 1], off[j:j + 1], ref, prob1)
-    # planted needles, every unit.  A needle is aligned with one window query only, and where several needles of
-    # a head share that row its attention is split, so a few fall short of the cut at this scale (the oracle pins
-    # the strict form on small cases).  Under heavy-tailed key scales or average pooling other keys pass the
-    # needles by design of the workload; there the oracle comparison above is the check.
-    if census and not cfg.heavy_tail and cfg.pool_kind == 1:
+        # needles as a parity statement: the GPU drops exactly the needles the oracle drops on its own scores
+        # (none, except where a head's budget is too small for them or heavy-tailed keys out-score them)
+        lost_gpu = dropped_needles(cfg, b["needles"][j], idx[j], off[j])
+        lost_ref = dropped_needles(cfg, b["needles"][j], ref["idx"][0], ref["offsets"][0])
+        if lost_gpu != lost_ref:       # allowed only inside the near-tie band of the head's k-th score
+            for g, t in sorted(lost_gpu ^ lost_ref):
+                e = int(ref["budgets"][0, g]) - cfg.window
+                kth = np.sort(sc[0, g])[::-1][e - 1]
+                print(f"needle {t} of unit {j} head {g}: oracle score {sc[0, g, t]:.6g}, k-th score {kth:.6g}")
+                assert abs(sc[0, g, t] - kth) <= SCORE_RTOL * abs(kth), (j, g, t)
+    # planted needles, every unit: strict.  Every needle's query row points away from the sink and serves one needle
+    # only (inputs.make_unit), so each needle holds a large share of its row's attention and must be kept wherever the
+    # head's budget covers all needle neighbourhoods.  Under heavy-tailed key scales other keys out-score the needles
+    # by design of the workload; there the statement is the parity one above (the GPU drops what the oracle drops).
+    if census and not cfg.heavy_tail:
         planted, kept, lost = needle_census(cfg, b, idx, bud, off)
-        assert kept >= 0.99 * planted, (kept, planted, lost[:8])
+        assert kept == planted, (kept, planted, lost[:8])
     del b, out
     torch.cuda.empty_cache()
 
