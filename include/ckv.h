@@ -13,18 +13,24 @@
  *     `_host`.  `shape` and `params` are HOST structs read before the call returns.
  *   - The caller owns every buffer.  The library allocates no device memory and
  *     keeps no per-call state; work space is passed in (`ws`, `ws_bytes`, at
- *     least ckv_workspace_bytes(), 256-byte aligned).
+ *     least ckv_workspace_bytes(), 256-byte aligned).  What the library does keep,
+ *     per process: the diagnostic settings of ckv_set_score_path and ckv_set_tunable
+ *     (results do not depend on them), a launch counter, and per-device constants it
+ *     looks up once (driver entry point, resident CTAs, the address of the fixed scratch);
+ *     per calling thread: the event pair of ckv_set_scan_events.
  *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL is
  *     the default stream) and return after the last launch was queued.
  *   - Errors are return codes.  Argument errors are found on the host before
  *     anything is launched (CKV_ERR_INVALID_ARG / UNSUPPORTED / WORKSPACE); a CUDA
  *     launch error gives CKV_ERR_CUDA.  A device-side wait that ran out of its
- *     time limit (2 s) is recorded in the work space's status word and read back
- *     with ckv_device_status().
+ *     time limit (2 s unless changed with ckv_set_tunable) is recorded in the work
+ *     space's status word, stays there over later calls, and is read back -- and
+ *     cleared -- by ckv_device_status().
  *   - Preconditions that are not checked: inputs are finite, head_w >= 0.
  *   - Layouts: q_win [Nu, H, W, d], k and v [Nu, Hkv, L, d]; the last dimension is
  *     contiguous and the other strides are given in ELEMENTS in ckv_shape; every row
- *     must start on a 16-byte boundary.  All outputs are dense.
+ *     must start on a 16-byte boundary; a stride of zero over an extent above one (a
+ *     broadcast view) is refused.  All outputs are dense.
  */
 #ifndef CKV_H_
 #define CKV_H_
@@ -88,10 +94,26 @@ typedef struct {
   int32_t units_per_prompt; /* with global_alpha: units [s N, (s+1) N) of the call belong to prompt s (its layers);
                                N >= 1 divides n_units.  Ignored otherwise (0 allowed) */
   int32_t reserved_;        /* set to 0 */
+  /* The threshold table as the paper indexes it (Sec. 4.3; Alg. 1 (D)): tau = T_gate[l, b_ent, b_ppl, B_l].
+     A non-null gate_coords switches it on.  `sens` is then the dense table
+     [n_gate_layers][n_buckets][n_ppl_bins][n_budget_levels] fp32 shared by all units (sens_stride_unit must be 0),
+     n_buckets counts the entropy bins (20 in the paper, with 4 perplexity bins), b_ent is the unit's entropy bin as
+     above, and gate_coords [Nu,3] int32 (DEVICE pointer; a HOST pointer for ckv_compress_host) gives per unit the
+     layer row l, the perplexity bin b_ppl of its prompt -- the caller's: Eq. 7's perplexity needs the language
+     model's logits -- and the index of its budget level.  Coordinates outside the table are clamped into it. */
+  int32_t n_gate_layers;    /* >= 1 with gate_coords; table rows along the layer axis (ckv_gate_depth_map_host maps a
+                               table compiled for another depth) */
+  int32_t n_ppl_bins;       /* >= 1 with gate_coords */
+  int32_t n_budget_levels;  /* >= 1 with gate_coords */
+  int32_t reserved2_;       /* set to 0 */
+  const int32_t* gate_coords;
 } ckv_params;
 
 /* Bytes of work space any entry point needs for this problem (0 on invalid arguments). */
 size_t ckv_workspace_bytes(const ckv_shape* shape, const ckv_params* params);
+/* Bytes that ckv_score alone needs: the leading sections of that work space (0 on invalid arguments).  This is
+ * also what a problem must fit into for ckv_score_noalloc. */
+size_t ckv_score_workspace_bytes(const ckv_shape* shape, const ckv_params* params);
 
 /*
  * Window-score scan and head-table weighting (Sec. 3 softmax; Eq. 4's window mass alpha; Eq. 6's
@@ -246,8 +268,9 @@ ckv_status ckv_compress_host(const ckv_shape* shape, const ckv_params* params, c
  *
  * The scratch is a fixed array of CKV_NOALLOC_SCRATCH_BYTES bytes in the library's own device
  * image: every GPU on which the library is loaded holds it from load until the process exits.
- * Problems whose ckv_workspace_bytes() exceeds that size are refused with CKV_ERR_WORKSPACE before
- * anything is launched (use ckv_score with a caller-owned work space for those).
+ * Only the sections of the work space that the score stage uses count against that size (a little over half
+ * of ckv_workspace_bytes(); about 7.5 MB per unit of 32 query heads at L = 32768); larger problems are refused
+ * with CKV_ERR_WORKSPACE before anything is launched (use ckv_score with a caller-owned work space for those).
  *   - Nothing is allocated or freed, by the CUDA runtime or otherwise.  The first call on a device
  *     looks up the array's device address (one runtime query, remembered per device); make that
  *     first call outside any stream capture.
@@ -255,8 +278,8 @@ ckv_status ckv_compress_host(const ckv_shape* shape, const ckv_params* params, c
  *     entry point clears the few words that must start at zero.  Two calls whose kernels can run at
  *     the same time on one device (different streams without an ordering between them) race on it:
  *     serialise them.
- *   - The device status word lives inside the array, so ckv_device_status() cannot report on this
- *     variant.
+ *   - The device status word lives inside the array: ckv_device_status(NULL, stream) reads it on the
+ *     current device.
  * Arguments, layouts, outputs and the remaining error codes are those of ckv_score.
  */
 #define CKV_NOALLOC_SCRATCH_BYTES (16u << 20)
@@ -264,8 +287,10 @@ ckv_status ckv_score_noalloc(const ckv_shape* shape, const ckv_params* params, c
                              const void* k, const float* head_w, float* scores, float* colmass,
                              void* stream);
 
-/* Synchronises `stream` and returns the status word device code wrote into `ws` (CKV_OK or
- * CKV_ERR_TIMEOUT), or CKV_ERR_CUDA if the stream is in error. */
+/* Synchronises `stream` and returns what device code recorded in the status word of `ws` since the last
+ * such call (CKV_OK or CKV_ERR_TIMEOUT), or CKV_ERR_CUDA if the stream is in error.  A recorded code survives
+ * later calls on the work space until this function reports it, which also clears it.  ws == NULL reads the
+ * fixed scratch of ckv_score_noalloc on the current device.  Work space that no call has used yet reads CKV_OK. */
 ckv_status ckv_device_status(const void* ws, void* stream);
 
 /* Diagnostic switch for the window-score scan: 0 = automatic (tensor-core kernel for bf16 inputs with
@@ -277,7 +302,8 @@ int ckv_set_score_path(int path);
 /* Timing hook: when both are non-null cudaEvent_t handles (created with timing enabled, owned by the
  * caller), every later ckv_score / ckv_compress call that runs the tensor-core scan records
  * start_event just before and stop_event just after that kernel's launch, on the call's stream, so
- * that the scan can be timed inside a fused call.  Pass nulls to switch it off.  Process-wide. */
+ * that the scan can be timed inside a fused call.  Pass nulls to switch it off.  The pair belongs to the calling
+ * thread: calls made from other threads are not affected and record nothing. */
 void ckv_set_scan_events(void* start_event, void* stop_event);
 
 /* Diagnostic knobs of the tensor-core scan (process-wide; the scores do not depend on them):
@@ -292,7 +318,10 @@ void ckv_set_scan_events(void* start_event, void* stop_event);
  *                    0: always write per-head column sums;
  *   "pdl"            1 (default): the counting, selection and gather kernels are launched with programmatic
  *                    stream serialisation, so each is scheduled while its predecessor drains and waits on the
- *                    device for it to complete; 0: ordinary launches.
+ *                    device for it to complete; 0: ordinary launches;
+ *   "wait_limit_us"  time limit of every bounded device-side wait in microseconds (default 2000000).  A wait
+ *                    that runs out makes its kernel wind down and records CKV_ERR_TIMEOUT in the status word;
+ *                    the outputs of that call are then incomplete.
  * Returns the previous value, or -1 for an unknown name or a value out of range. */
 int ckv_set_tunable(const char* name, int value);
 
@@ -303,6 +332,14 @@ int64_t ckv_kernel_launches(void);
  * shares in [f, n], f*hkv <= P <= n*hkv), exposed so that it can be checked without a GPU.
  * Returns 0 on success. */
 int ckv_allocate_rows_host(int hkv, int64_t n, int64_t f, int64_t P, const int64_t* demands, int64_t* out);
+
+/* Host-only: a table compiled for n_src layers ([n_src][row_elems] fp32, e.g. the gate table with row_elems =
+ * n_buckets * n_ppl_bins * n_budget_levels, or the head table with row_elems = H) mapped to a model of n_dst
+ * layers by relative depth (the paper's appendix on cross-architecture use: a monotone depth mapping by
+ * relative-depth interpolation): target layer l takes the linear interpolation of the source rows around
+ * position l (n_src - 1) / (n_dst - 1); first and last layers map onto first and last, equal depths give a copy.
+ * dst [n_dst][row_elems].  Returns 0 on success, 1 on invalid arguments. */
+int ckv_gate_depth_map_host(const float* src, int n_src, int n_dst, int64_t row_elems, float* dst);
 
 const char* ckv_status_string(ckv_status status);
 int ckv_version(void);

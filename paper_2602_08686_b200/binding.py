@@ -38,7 +38,9 @@ class ckv_params(C.Structure):
                                          "n_buckets", "bucket_override")] + \
                [(n, C.c_int64) for n in ("head_w_stride_unit", "sens_stride_unit")] + \
                [("value_norm", C.c_int32), ("value_norm_eps", C.c_float), ("shared_elastic", C.c_int32),
-                ("global_alpha", C.c_int32), ("units_per_prompt", C.c_int32), ("reserved_", C.c_int32)]
+                ("global_alpha", C.c_int32), ("units_per_prompt", C.c_int32), ("reserved_", C.c_int32),
+                ("n_gate_layers", C.c_int32), ("n_ppl_bins", C.c_int32), ("n_budget_levels", C.c_int32),
+                ("reserved2_", C.c_int32), ("gate_coords", C.c_void_p)]
 
 
 _lib = None
@@ -56,6 +58,8 @@ def lib() -> C.CDLL:
         shp, prm = C.POINTER(ckv_shape), C.POINTER(ckv_params)
         L.ckv_workspace_bytes.restype = sz
         L.ckv_workspace_bytes.argtypes = [shp, prm]
+        L.ckv_score_workspace_bytes.restype = sz
+        L.ckv_score_workspace_bytes.argtypes = [shp, prm]
         L.ckv_staging_bytes.restype = sz
         L.ckv_staging_bytes.argtypes = [shp, prm]
         L.ckv_score.argtypes = [shp, prm, vp, vp, fp, fp, fp, vp, sz, vp]
@@ -72,6 +76,7 @@ def lib() -> C.CDLL:
         L.ckv_compress.argtypes = [shp, prm, vp, vp, vp, fp, fp, vp, vp, i32p, i32p, i32p, fp, i32p, fp, vp, sz, vp]
         L.ckv_compress_host.argtypes = [shp, prm, vp, vp, vp, fp, fp, vp, vp, i32p, i32p, i32p, vp, sz, vp, sz, vp]
         L.ckv_device_status.argtypes = [vp, vp]
+        L.ckv_gate_depth_map_host.argtypes = [fp, C.c_int, C.c_int, C.c_int64, fp]
         L.ckv_set_scan_events.argtypes = [vp, vp]
         L.ckv_set_scan_events.restype = None
         L.ckv_set_tunable.argtypes = [C.c_char_p, C.c_int]
@@ -133,6 +138,11 @@ class Params:
     shared_elastic: bool = False
     global_alpha: bool = False
     units_per_prompt: int = 1
+    # the four-axis gate table T_gate[layer, entropy bin, perplexity bin, budget level] (used when make_params is
+    # given gate_coords); n_buckets is then the number of entropy bins
+    n_gate_layers: int = 0
+    n_ppl_bins: int = 1
+    n_budget_levels: int = 1
 
 
 def _dtype_code(t: torch.Tensor) -> int:
@@ -153,12 +163,26 @@ def make_shape(q: torch.Tensor, k: torch.Tensor) -> ckv_shape:
                      k.stride(0), k.stride(1), k.stride(2))
 
 
-def make_params(p: Params, head_w: torch.Tensor | None, sens: torch.Tensor | None, H: int = 0) -> ckv_params:
+def make_params(p: Params, head_w: torch.Tensor | None, sens: torch.Tensor | None, H: int = 0,
+                gate_coords: torch.Tensor | None = None) -> ckv_params:
+    """Parameter struct.  With gate_coords ([Nu,3] int32: layer row, perplexity bin, budget level per unit; on the
+    device, or on the host for ckv_compress_host) `sens` is the dense table [n_gate_layers, n_buckets, n_ppl_bins,
+    n_budget_levels]; the struct keeps a reference to the tensor."""
     hw_stride = 0 if head_w is None or head_w.dim() == 1 else head_w.stride(0)
-    se_stride = 0 if sens is None or sens.dim() == 1 else sens.stride(0)
-    return ckv_params(p.pool_kind, p.pool_size, p.budget_per_head, p.floor_per_head, p.n_buckets,
-                      p.bucket_override, hw_stride, se_stride, int(p.value_norm), float(p.value_norm_eps), int(p.shared_elastic), int(p.global_alpha),
-                      int(p.units_per_prompt), 0)
+    se_stride = 0 if sens is None or sens.dim() == 1 or gate_coords is not None else sens.stride(0)
+    if gate_coords is not None:
+        if gate_coords.dtype != torch.int32 or not gate_coords.is_contiguous() or gate_coords.shape[-1] != 3:
+            raise ValueError("gate_coords must be a contiguous int32 tensor [Nu, 3]")
+        if sens is not None and (not sens.is_contiguous() or sens.numel() != p.n_gate_layers * p.n_buckets *
+                                 p.n_ppl_bins * p.n_budget_levels):
+            raise ValueError("the gate table must be dense [n_gate_layers, n_buckets, n_ppl_bins, n_budget_levels]")
+    out = ckv_params(p.pool_kind, p.pool_size, p.budget_per_head, p.floor_per_head, p.n_buckets,
+                     p.bucket_override, hw_stride, se_stride, int(p.value_norm), float(p.value_norm_eps),
+                     int(p.shared_elastic), int(p.global_alpha), int(p.units_per_prompt), 0,
+                     int(p.n_gate_layers) if gate_coords is not None else 0, int(p.n_ppl_bins),
+                     int(p.n_budget_levels), 0, None if gate_coords is None else gate_coords.data_ptr())
+    out._keep = gate_coords
+    return out
 
 
 def _ptr(t):
@@ -170,6 +194,22 @@ def _stream(stream=None):
     return C.c_void_p(s.cuda_stream)
 
 
+def _check_kv(shape: ckv_shape, t: torch.Tensor, name: str) -> None:
+    """k and v share one set of strides in ckv_shape: a tensor laid out differently would be read wrongly."""
+    want_shape = (shape.n_units, shape.n_kv_heads, shape.seq_len, shape.head_dim)
+    if tuple(t.shape) != want_shape or _dtype_code(t) != shape.dtype or t.stride(3) != 1:
+        raise ValueError(f"{name} must be {want_shape} in the dtype of the shape struct, last dimension contiguous")
+    for dim, want in enumerate((shape.kv_stride_unit, shape.kv_stride_head, shape.kv_stride_tok)):
+        if t.shape[dim] > 1 and t.stride(dim) != want:
+            raise ValueError(f"{name} has stride {t.stride(dim)} in dimension {dim}; the shape struct says {want} "
+                             "(k and v must be laid out alike)")
+
+
+def _check_dense(t: torch.Tensor, name: str) -> None:
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be dense")
+
+
 def _check(status: int, what: str):
     if status != OK:
         raise CkvError(status, what)
@@ -177,6 +217,10 @@ def _check(status: int, what: str):
 
 def ckv_workspace_bytes(shape: ckv_shape, params: ckv_params) -> int:
     return int(lib().ckv_workspace_bytes(C.byref(shape), C.byref(params)))
+
+
+def ckv_score_workspace_bytes(shape: ckv_shape, params: ckv_params) -> int:
+    return int(lib().ckv_score_workspace_bytes(C.byref(shape), C.byref(params)))
 
 
 def ckv_staging_bytes(shape: ckv_shape, params: ckv_params) -> int:
@@ -216,6 +260,7 @@ def ckv_budget(shape, params, scores, colmass, sens, budgets, offsets, bucket, e
 
 
 def ckv_vnorm(shape, params, v, rho, scores, ws, stream=None):
+    _check_kv(shape, v, "v")
     _check(lib().ckv_vnorm(C.byref(shape), C.byref(params), _ptr(v), _ptr(rho), _ptr(scores), _ptr(ws), ws.numel(),
                            _stream(stream)), "ckv_vnorm")
 
@@ -239,6 +284,11 @@ def ckv_attend(shape, params, q_dec, k, v, out, lse, ws, budgets=None, offsets=N
     """Attention of the decode queries q_dec [Nu,H,n_dec,d] over all rows of k, v, or over the gathered rows when
     budgets and offsets are given."""
     compressed = budgets is not None
+    _check_dense(q_dec, "q_dec")
+    if not compressed:
+        _check_kv(shape, k, "k"), _check_kv(shape, v, "v")
+    else:
+        _check_dense(k, "k_out"), _check_dense(v, "v_out")
     _check(lib().ckv_attend(C.byref(shape), C.byref(params), _ptr(q_dec), int(q_dec.shape[2]), _ptr(k), _ptr(v),
                             int(compressed), _ptr(budgets), _ptr(offsets), _ptr(out), _ptr(lse), _ptr(ws), ws.numel(),
                             _stream(stream)), "ckv_attend")
@@ -254,12 +304,16 @@ def ckv_select(shape, params, scores, budgets, offsets, indices, ws, stream=None
 
 
 def ckv_gather(shape, params, k, v, indices, offsets, k_out, v_out, stream=None):
+    _check_kv(shape, k, "k"), _check_kv(shape, v, "v")
+    _check_dense(k_out, "k_out"), _check_dense(v_out, "v_out")
     _check(lib().ckv_gather(C.byref(shape), C.byref(params), _ptr(k), _ptr(v), _ptr(indices), _ptr(offsets),
                             _ptr(k_out), _ptr(v_out), _stream(stream)), "ckv_gather")
 
 
 def ckv_compress(shape, params, q_win, k, v, head_w, sens, k_out, v_out, indices, budgets, offsets, ws,
                  scores=None, bucket=None, entropy=None, stream=None):
+    _check_kv(shape, k, "k"), _check_kv(shape, v, "v")
+    _check_dense(k_out, "k_out"), _check_dense(v_out, "v_out")
     _check(lib().ckv_compress(C.byref(shape), C.byref(params), _ptr(q_win), _ptr(k), _ptr(v), _ptr(head_w),
                               _ptr(sens), _ptr(k_out), _ptr(v_out), _ptr(indices), _ptr(budgets), _ptr(offsets),
                               _ptr(scores), _ptr(bucket), _ptr(entropy), _ptr(ws), ws.numel(), _stream(stream)),
@@ -275,8 +329,21 @@ def ckv_compress_host(shape, params, q_win, k, v, head_w, sens, k_out, v_out, in
                                    _stream(stream)), "ckv_compress_host")
 
 
-def ckv_device_status(ws, stream=None) -> int:
+def ckv_device_status(ws=None, stream=None) -> int:
+    """What device code recorded in the work space's status word since the last such call (reading clears it);
+    ``ws=None`` reads the fixed scratch of ckv_score_noalloc on the current device."""
     return int(lib().ckv_device_status(_ptr(ws), _stream(stream)))
+
+
+def ckv_gate_depth_map_host(table: torch.Tensor, n_dst: int) -> torch.Tensor:
+    """A host table [n_src, ...] (fp32) compiled for n_src layers, mapped to n_dst layers by relative depth."""
+    src = table.detach().cpu().contiguous().float()
+    n_src = src.shape[0]
+    row = src[0].numel() if src.dim() > 1 else 1
+    dst = torch.empty((n_dst,) + tuple(src.shape[1:]), dtype=torch.float32)
+    if lib().ckv_gate_depth_map_host(_ptr(src), n_src, int(n_dst), row, _ptr(dst)) != 0:
+        raise ValueError("ckv_gate_depth_map_host: invalid arguments")
+    return dst
 
 
 def ckv_allocate_rows_host(n: int, f: int, P: int, demands) -> list[int]:
@@ -291,10 +358,11 @@ def ckv_allocate_rows_host(n: int, f: int, P: int, demands) -> list[int]:
 
 
 # ------------------------------------------------------------------------------------ convenience
-def compress(q_win, k, v, head_w, sens, p: Params, want_scores: bool = False, ws=None, stream=None):
+def compress(q_win, k, v, head_w, sens, p: Params, want_scores: bool = False, ws=None, stream=None,
+             gate_coords=None):
     """Allocates the outputs and the work space with torch and runs ckv_compress."""
     shape = make_shape(q_win, k)
-    params = make_params(p, head_w, sens)
+    params = make_params(p, head_w, sens, gate_coords=gate_coords)
     dev = k.device
     Nu, Hkv = shape.n_units, shape.n_kv_heads
     rows = rows_per_unit(shape, params)

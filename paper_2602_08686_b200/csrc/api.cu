@@ -1,4 +1,5 @@
 // Host side of the C ABI: argument validation, work-space layout and the launch sequences.
+#include <algorithm>
 #include <atomic>
 #include <string>
 #include <cstring>
@@ -13,10 +14,13 @@ static std::atomic<int> g_score_path{0};  // 0 = automatic, 1 = plain kernels, 2
 static std::atomic<int> g_pdl{1};         // 1: the kernels after the pooling kernel use programmatic dependent launch
 bool pdl_enabled() { return g_pdl.load(std::memory_order_relaxed) != 0; }
 static std::atomic<int> g_group_fuse{1};  // 1: the scan writes per-group maxima and masses where it can
-static std::atomic<cudaEvent_t> g_scan_start{nullptr}, g_scan_stop{nullptr};  // see ckv_set_scan_events
+static std::atomic<unsigned long long> g_wait_limit_ns{2000000000ull};   // bound of every device-side wait
+unsigned long long wait_limit_ns() { return g_wait_limit_ns.load(std::memory_order_relaxed); }
+static thread_local cudaEvent_t t_scan_start = nullptr, t_scan_stop = nullptr;  // see ckv_set_scan_events
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
 static size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+static ckv_status noalloc_scratch(char** out);   // device address of the fixed scratch (end of this file)
 
 WsLayout ws_layout(const ckv_shape& s, const ckv_params& p) {
   WsLayout w{};
@@ -24,21 +28,29 @@ WsLayout ws_layout(const ckv_shape& s, const ckv_params& p) {
   const size_t n = L - W;
   w.nblk = (int)((L + kPlainKeysPerBlock - 1) / kPlainKeysPerBlock);
   size_t o = 0;
+  // what the score stage touches comes first, so that its extent alone decides whether a problem fits a small
+  // fixed scratch (ckv_score_noalloc)
   w.status = o, o += 256;
-  if (s.dtype == CKV_BF16) w.tc_flags = o, o = align_up(o + tc_layout(s).flag_bytes);   // behind the status words: one memset clears both
+  if (s.dtype == CKV_BF16) w.tc_flags = o, o = align_up(o + tc_layout(s).flag_bytes);   // behind the status words: one kernel clears both
   w.csum = o, o = align_up(o + Nu * H * L * sizeof(float));
   w.part = o, o = align_up(o + Nu * H * W * (size_t)w.nblk * sizeof(float2));
   w.stat = o, o = align_up(o + Nu * H * W * sizeof(float2));
+  {
+    const BudgetLayout b = budget_layout(s);
+    w.ent_part = o, o = align_up(o + b.ent_bytes);
+    w.bud_done = o, o = align_up(o + b.done_bytes);
+    if (s.dtype == CKV_BF16) {
+      const TcLayout t = tc_layout(s);
+      w.tc_part = o, o = align_up(o + t.part_bytes);
+      w.tc_stat = o, o = align_up(o + t.stat_bytes);
+    }
+    w.score_extent = o;
+    w.cnt_part = o, o = align_up(o + b.cnt_bytes);
+  }
   w.colmass = o, o = align_up(o + Nu * L * sizeof(float));
   w.scores = o, o = align_up(o + Nu * Hkv * (n ? n : 1) * sizeof(float));
   w.bucket = o, o = align_up(o + Nu * sizeof(int32_t));
   w.entropy = o, o = align_up(o + Nu * sizeof(float));
-  {
-    const BudgetLayout b = budget_layout(s);
-    w.ent_part = o, o = align_up(o + b.ent_bytes);
-    w.cnt_part = o, o = align_up(o + b.cnt_bytes);
-    w.bud_done = o, o = align_up(o + b.done_bytes);
-  }
   w.pmass = o, o = align_up(o + (p.global_alpha ? Nu / (size_t)p.units_per_prompt * L * sizeof(float) : 0));
   {
     const size_t slots = Nu * Hkv * (size_t)attend_slices(s) * kAttendMaxRows;
@@ -47,11 +59,6 @@ WsLayout ws_layout(const ckv_shape& s, const ckv_params& p) {
   }
   w.vn_part = o, o = align_up(o + Nu * Hkv * ((L + kVnormRows - 1) / kVnormRows) * sizeof(float));
   w.vn_rho = o, o = align_up(o + (p.value_norm ? Nu * Hkv * L * sizeof(float) : 0));
-  if (s.dtype == CKV_BF16) {
-    const TcLayout t = tc_layout(s);
-    w.tc_part = o, o = align_up(o + t.part_bytes);
-    w.tc_stat = o, o = align_up(o + t.stat_bytes);
-  }
   w.total = o;
   return w;
 }
@@ -74,6 +81,11 @@ static ckv_status check_shape(const ckv_shape* s) {
   for (int64_t st : strides)
     if (st < 0 || (st * esz) % 16) return CKV_ERR_INVALID_ARG;
   if (s->q_stride_row < kHeadDim || s->kv_stride_tok < kHeadDim) return CKV_ERR_INVALID_ARG;
+  // a zero stride over more than one element (a broadcast view) is refused: the tensor maps of the scan cannot
+  // describe it, and no caller of a retention pass has two units or heads that share their rows
+  if ((s->n_units > 1 && (s->q_stride_unit == 0 || s->kv_stride_unit == 0)) ||
+      (s->n_q_heads > 1 && s->q_stride_head == 0) || (s->n_kv_heads > 1 && s->kv_stride_head == 0))
+    return CKV_ERR_INVALID_ARG;
   return CKV_OK;
 }
 
@@ -90,6 +102,14 @@ static ckv_status check_params(const ckv_shape* s, const ckv_params* p) {
   if (p->units_per_prompt < 0) return CKV_ERR_INVALID_ARG;
   if (p->global_alpha && (p->units_per_prompt < 1 || s->n_units % p->units_per_prompt)) return CKV_ERR_INVALID_ARG;
   if (!(p->value_norm_eps >= 0.f) || !(p->value_norm_eps < 3.0e38f)) return CKV_ERR_INVALID_ARG;
+  if (p->n_gate_layers < 0 || p->n_ppl_bins < 0 || p->n_budget_levels < 0) return CKV_ERR_INVALID_ARG;
+  if (p->gate_coords) {   // the four-axis gate table: one dense table for all units
+    if (p->n_gate_layers < 1 || p->n_ppl_bins < 1 || p->n_budget_levels < 1 || p->sens_stride_unit != 0)
+      return CKV_ERR_INVALID_ARG;
+    if (!aligned(p->gate_coords, 4)) return CKV_ERR_INVALID_ARG;
+    if ((int64_t)p->n_gate_layers * p->n_buckets * p->n_ppl_bins * p->n_budget_levels > (int64_t)1 << 30)
+      return CKV_ERR_UNSUPPORTED;
+  }
   if (p->budget_per_head < s->seq_len) {
     if (p->budget_per_head < s->window) return CKV_ERR_INVALID_ARG;
     if (p->floor_per_head > p->budget_per_head - s->window) return CKV_ERR_INVALID_ARG;
@@ -123,6 +143,28 @@ static bool all_aligned4(std::initializer_list<const void*> ps) {
     if ((expr) != cudaSuccess) return CKV_ERR_CUDA;  \
   } while (0)
 
+// Word kStatusMagicWord of the status section says that words 0..7 (the status code and the waits that were in
+// progress when it was set) are meaningful; a work space seen for the first time has them cleared.  The words
+// behind them (counters, the scan's flags and queues) are cleared on every call.
+constexpr int kStatusMagicWord = 63;
+constexpr int kStatusMagic = 0x434b5631;
+__global__ void ws_reset_kernel(int* status, size_t n_flag_words) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x, step = (size_t)gridDim.x * blockDim.x;
+  if (i == 0 && status[kStatusMagicWord] != kStatusMagic) {
+    for (int w = 0; w < 8; ++w) status[w] = 0;
+    status[kStatusMagicWord] = kStatusMagic;
+  }
+  if (i >= 8 && i < (size_t)kStatusMagicWord) status[i] = 0;
+  int* flags = status + 64;
+  for (size_t w = i; w < n_flag_words; w += step) flags[w] = 0;
+}
+static cudaError_t launch_ws_reset(int* status, size_t n_flag_words, cudaStream_t st) {
+  const int blocks = (int)std::min<size_t>(64, (n_flag_words + 255) / 256 + 1);
+  ws_reset_kernel<<<blocks, 256, 0, st>>>(status, n_flag_words);
+  count_launch();
+  return cudaGetLastError();
+}
+
 static ckv_status score_impl(const ckv_shape& s, const ckv_params& p, const void* q, const void* k,
                              const float* head_w, float* scores, float* colmass, char* ws, cudaStream_t st) {
   const WsLayout w = ws_layout(s, p);
@@ -130,10 +172,11 @@ static ckv_status score_impl(const ckv_shape& s, const ckv_params& p, const void
   const bool tc_ok = score_tc_supported(s) && s.seq_len >= 128;
   if (path == 2 && !tc_ok) return CKV_ERR_UNSUPPORTED;
   const bool use_tc = tc_ok && path != 1;
-  // the status words and, behind them, the tensor-core scan's counters and run queues
-  CKV_CUDA(cudaMemsetAsync(ws + w.status, 0, 256 + (use_tc ? tc_layout(s).flag_bytes : 0), st));
+  // the scheduler words and, behind them, the tensor-core scan's counters and run queues start at zero; the
+  // status words keep a code that no ckv_device_status call has read yet
+  CKV_CUDA(launch_ws_reset(reinterpret_cast<int*>(ws + w.status), use_tc ? tc_layout(s).flag_bytes / sizeof(int) : 0, st));
   float* csum = reinterpret_cast<float*>(ws + w.csum);
-  const cudaEvent_t ev0 = g_scan_start.load(), ev1 = g_scan_stop.load();
+  const cudaEvent_t ev0 = t_scan_start, ev1 = t_scan_stop;
   int* marker = reinterpret_cast<int*>(ws + w.status) + kPathMarkerWord;   // who wrote the row statistics
   if (use_tc) {
     // grouped output where it applies: both arrays fit the per-head region (at least two heads per group)
@@ -169,12 +212,18 @@ size_t ckv_workspace_bytes(const ckv_shape* shape, const ckv_params* params) {
   return ws_layout(*shape, *params).total;
 }
 
+size_t ckv_score_workspace_bytes(const ckv_shape* shape, const ckv_params* params) {
+  if (check_shape(shape) != CKV_OK || check_params(shape, params) != CKV_OK) return 0;
+  return ws_layout(*shape, *params).score_extent;
+}
+
 ckv_status ckv_score(const ckv_shape* shape, const ckv_params* params, const void* q_win, const void* k,
                      const float* head_w, float* scores, float* colmass, void* ws, size_t ws_bytes, void* stream) {
   CKV_TRY(check_shape(shape));
   CKV_TRY(check_params(shape, params));
   if (!all_aligned16({q_win, k}) || !all_aligned4({head_w, scores, colmass})) return CKV_ERR_INVALID_ARG;
-  CKV_TRY(check_ws(shape, params, ws, ws_bytes));
+  // the score stage alone uses the leading sections of the work space
+  if (!ws || !aligned(ws, 256) || ws_bytes < ws_layout(*shape, *params).score_extent) return CKV_ERR_WORKSPACE;
   return score_impl(*shape, *params, q_win, k, head_w, scores, colmass, (char*)ws, (cudaStream_t)stream);
 }
 
@@ -331,6 +380,7 @@ ckv_status ckv_compress(const ckv_shape* shape, const ckv_params* params, const 
 struct Staging {
   size_t q, k, v, head_w, sens, k_out, v_out, indices, budgets, offsets, total;
   size_t q_b, kv_b, hw_b, sens_b, out_b, idx_b, bud_b, off_b;
+  size_t coords, coords_b;   // gate coordinates [Nu,3] (only with the four-axis gate table)
 };
 static Staging staging_layout(const ckv_shape& s, const ckv_params& p) {
   Staging g{};
@@ -341,6 +391,8 @@ static Staging staging_layout(const ckv_shape& s, const ckv_params& p) {
   g.kv_b = Nu * Hkv * L * d * esz;
   g.hw_b = (p.head_w_stride_unit ? Nu : 1) * H * sizeof(float);
   g.sens_b = (p.sens_stride_unit ? Nu : 1) * (size_t)p.n_buckets * sizeof(float);
+  if (p.gate_coords) g.sens_b = (size_t)p.n_gate_layers * p.n_buckets * p.n_ppl_bins * p.n_budget_levels * sizeof(float);
+  g.coords_b = p.gate_coords ? Nu * 3 * sizeof(int32_t) : 0;
   g.out_b = Nu * rows * d * esz;
   g.idx_b = Nu * rows * sizeof(int32_t);
   g.bud_b = Nu * Hkv * sizeof(int32_t);
@@ -356,6 +408,7 @@ static Staging staging_layout(const ckv_shape& s, const ckv_params& p) {
   g.indices = o, o = align_up(o + g.idx_b);
   g.budgets = o, o = align_up(o + g.bud_b);
   g.offsets = o, o = align_up(o + g.off_b);
+  g.coords = o, o = align_up(o + g.coords_b);
   g.total = o;
   return g;
 }
@@ -395,6 +448,10 @@ ckv_status ckv_compress_host(const ckv_shape* shape, const ckv_params* params, c
   CKV_CUDA(cudaMemcpyAsync(d + g.v, v_host, g.kv_b, cudaMemcpyHostToDevice, st));
   CKV_CUDA(cudaMemcpyAsync(d + g.head_w, head_w_host, g.hw_b, cudaMemcpyHostToDevice, st));
   CKV_CUDA(cudaMemcpyAsync(d + g.sens, sens_host, g.sens_b, cudaMemcpyHostToDevice, st));
+  if (params->gate_coords) {
+    CKV_CUDA(cudaMemcpyAsync(d + g.coords, params->gate_coords, g.coords_b, cudaMemcpyHostToDevice, st));
+    p.gate_coords = reinterpret_cast<const int32_t*>(d + g.coords);
+  }
   CKV_TRY(ckv_compress(&s, &p, d + g.q, d + g.k, d + g.v, (const float*)(d + g.head_w), (const float*)(d + g.sens),
                        d + g.k_out, d + g.v_out, (int32_t*)(d + g.indices), (int32_t*)(d + g.budgets),
                        (int32_t*)(d + g.offsets), nullptr, nullptr, nullptr, ws, ws_bytes, stream));
@@ -408,12 +465,25 @@ ckv_status ckv_compress_host(const ckv_shape* shape, const ckv_params* params, c
 }
 
 ckv_status ckv_device_status(const void* ws, void* stream) {
-  if (!ws) return CKV_ERR_WORKSPACE;
-  int32_t word = 0;
-  if (cudaMemcpyAsync(&word, ws, sizeof(word), cudaMemcpyDeviceToHost, (cudaStream_t)stream) != cudaSuccess)
+  if (!ws) {   // the fixed scratch of ckv_score_noalloc on the current device
+    char* scratch = nullptr;
+    if (noalloc_scratch(&scratch) != CKV_OK) return CKV_ERR_CUDA;
+    ws = scratch;
+  }
+  if (!aligned(ws, 256)) return CKV_ERR_WORKSPACE;
+  int32_t words[2] = {0, 0};   // the code, and the magic word that says the code is meaningful
+  cudaStream_t st = (cudaStream_t)stream;
+  const char* base = static_cast<const char*>(ws);
+  if (cudaMemcpyAsync(&words[0], base, sizeof(int32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaMemcpyAsync(&words[1], base + kStatusMagicWord * sizeof(int32_t), sizeof(int32_t), cudaMemcpyDeviceToHost,
+                      st) != cudaSuccess)
     return CKV_ERR_CUDA;
-  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return CKV_ERR_CUDA;
-  return word == 0 ? CKV_OK : CKV_ERR_TIMEOUT;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return CKV_ERR_CUDA;
+  if (words[1] != kStatusMagic || words[0] == 0) return CKV_OK;   // never used by a call, or nothing recorded
+  // a recorded code is reported once: clear it (and the words that name the waits) for the calls that follow
+  if (cudaMemsetAsync(const_cast<char*>(base), 0, 8 * sizeof(int32_t), st) != cudaSuccess) return CKV_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return CKV_ERR_CUDA;
+  return CKV_ERR_TIMEOUT;
 }
 
 int ckv_set_score_path(int path) {
@@ -422,18 +492,37 @@ int ckv_set_score_path(int path) {
 }
 
 void ckv_set_scan_events(void* start_event, void* stop_event) {
-  g_scan_start.store((cudaEvent_t)start_event);
-  g_scan_stop.store((cudaEvent_t)stop_event);
+  t_scan_start = (cudaEvent_t)start_event;
+  t_scan_stop = (cudaEvent_t)stop_event;
 }
 
 int ckv_set_tunable(const char* name, int value) {
   if (!name) return -1;
   if (std::string(name) == "group_fuse") return g_group_fuse.exchange(value != 0 ? 1 : 0);
   if (std::string(name) == "pdl") return g_pdl.exchange(value != 0 ? 1 : 0);
+  if (std::string(name) == "wait_limit_us") {
+    if (value < 1) return -1;
+    return (int)(g_wait_limit_ns.exchange((unsigned long long)value * 1000ull) / 1000ull);
+  }
   return set_tc_tunable(name, value);
 }
 
 int64_t ckv_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int ckv_gate_depth_map_host(const float* src, int n_src, int n_dst, int64_t row_elems, float* dst) {
+  if (!src || !dst || n_src < 1 || n_dst < 1 || row_elems < 1) return 1;
+  for (int l = 0; l < n_dst; ++l) {
+    // position of target layer l on the source's layer axis, by relative depth
+    const double pos = n_dst > 1 ? (double)l * (n_src - 1) / (double)(n_dst - 1) : 0.0;
+    const int below = std::min((int)pos, n_src - 1), above = std::min(below + 1, n_src - 1);
+    const double frac = pos - below;
+    const float* a = src + (int64_t)below * row_elems;
+    const float* b = src + (int64_t)above * row_elems;
+    float* out = dst + (int64_t)l * row_elems;
+    for (int64_t c = 0; c < row_elems; ++c) out[c] = (float)((double)a[c] * (1.0 - frac) + (double)b[c] * frac);
+  }
+  return 0;
+}
 
 const char* ckv_status_string(ckv_status status) {
   switch (status) {
@@ -470,7 +559,6 @@ int ckv_allocate_rows_host(int hkv, int64_t n, int64_t f, int64_t P, const int64
 static __device__ __align__(256) unsigned char g_noalloc_scratch[CKV_NOALLOC_SCRATCH_BYTES];
 
 namespace ckv {
-constexpr int kMaxDevices = 64;
 static std::mutex g_noalloc_mutex;
 static void* g_noalloc_ptr[kMaxDevices] = {};
 
@@ -496,11 +584,12 @@ extern "C" ckv_status ckv_score_noalloc(const ckv_shape* shape, const ckv_params
   CKV_TRY(check_shape(shape));
   CKV_TRY(check_params(shape, params));
   if (!all_aligned16({q_win, k}) || !all_aligned4({head_w, scores, colmass})) return CKV_ERR_INVALID_ARG;
-  if (ws_layout(*shape, *params).total > (size_t)CKV_NOALLOC_SCRATCH_BYTES) return CKV_ERR_WORKSPACE;
+  if (ws_layout(*shape, *params).score_extent > (size_t)CKV_NOALLOC_SCRATCH_BYTES) return CKV_ERR_WORKSPACE;
   char* scratch = nullptr;
   CKV_TRY(noalloc_scratch(&scratch));
-  // score_impl zeroes the status word and the scan's counters before its kernels read them; the rest
-  // of the scratch is written before it is read, so what the previous call left behind is harmless.
+  // score_impl clears the scan's counters before its kernels read them and touches nothing beyond the score
+  // stage's sections; the rest of those is written before it is read, so what the previous call left behind
+  // is harmless.
   return score_impl(*shape, *params, q_win, k, head_w, scores, colmass, scratch, (cudaStream_t)stream);
 }
 #pragma GCC visibility pop

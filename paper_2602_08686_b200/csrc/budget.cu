@@ -119,7 +119,14 @@ __global__ void __launch_bounds__(kThreads) count_allocate(ckv_shape s, ckv_para
       int b = (int)floor(hn * (double)p.n_buckets);
       b = min(max(b, 0), p.n_buckets - 1);
       if (p.bucket_override >= 0) b = min(p.bucket_override, p.n_buckets - 1);
-      tau_s = sens[(int64_t)u * p.sens_stride_unit + b];
+      if (p.gate_coords) {   // Alg. 1 (D): tau = T_gate[l, b_ent, b_ppl, B_l]; coordinates held inside the table
+        const int32_t* c = p.gate_coords + (int64_t)u * 3;
+        const int l = min(max(c[0], 0), p.n_gate_layers - 1), bp = min(max(c[1], 0), p.n_ppl_bins - 1);
+        const int bb = min(max(c[2], 0), p.n_budget_levels - 1);
+        tau_s = sens[(((int64_t)l * p.n_buckets + b) * p.n_ppl_bins + bp) * p.n_budget_levels + bb];
+      } else {
+        tau_s = sens[(int64_t)u * p.sens_stride_unit + b];
+      }
       bucket_s = b, ent_s = ent, cnt_s = 0;
     }
   }

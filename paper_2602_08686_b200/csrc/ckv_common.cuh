@@ -15,6 +15,7 @@ constexpr int kEntSpan = 512;            // positions per entropy partial of the
 constexpr int kAttendMaxRows = 32;       // query rows (group size x decode queries) of the decode-side check
 constexpr int kVnormRows = 256;          // value rows per block sum of the value-norm stage
 constexpr int kCountSpan = 8192;         // scores per counting CTA of the budget stage
+constexpr int kMaxDevices = 64;          // devices the per-device caches of the host code cover
 
 // log2(e): the softmax is evaluated in base 2, x = (q.k) * log2(e) / sqrt(d)
 constexpr float kLog2e = 1.4426950408889634f;
@@ -40,6 +41,7 @@ struct WsLayout {
   size_t att_o;    // float [Nu, Hkv, slices, 32, 128]: per-slice partial results of the decode-side check
   size_t vn_part;  // float [Nu, Hkv, ceil(L / kVnormRows)] block sums of the value-row norms
   size_t vn_rho;   // float [Nu, Hkv, L]       value-norm ratios of the fused call (only with value_norm)
+  size_t score_extent;  // end of the sections the score stage uses (they come first)
   size_t total;
   int nblk;
 };
@@ -78,6 +80,8 @@ cudaError_t launch_score_tc(const ckv_shape& s, const void* q, const void* k, fl
 WsLayout ws_layout(const ckv_shape& s, const ckv_params& p);
 
 void count_launch(int n = 1);
+// Time limit of every bounded device-side wait, in nanoseconds (ckv_set_tunable "wait_limit_us"; default 2 s).
+unsigned long long wait_limit_ns();
 
 // Programmatic dependent launch between the small kernels that follow the scan: a kernel launched with
 // pdl_attribute() may be scheduled while its predecessor in the stream drains, and must call pdl_wait() before it

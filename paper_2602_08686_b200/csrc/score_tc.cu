@@ -10,8 +10,9 @@
 // A "chunk" is one (unit, KV head, block of 128 query rows); a "run" is a few consecutive key tiles of
 // a chunk.  CTAs take runs from two global queues (atomic counters), one per pass, in run order: P1
 // runs can always be taken; a P2 run can start once its chunk's statistics are final, which happens
-// shortly after the chunk's last P1 run, so the second read of a K tile usually comes from L2.  Results
-// do not depend on which CTA takes which run.  Warp roles:
+// shortly after the chunk's last P1 run.  By then the other CTAs have streamed far more than L2 retains, so
+// the second read of a K tile comes from HBM as well (L2 serves the query blocks and the partial statistics).
+// Results do not depend on which CTA takes which run.  Warp roles:
 //   warp 0       producer (one thread): hands runs to two "lanes" (the even and the odd sub-items),
 //                issues the TMA loads and describes every sub-item (one tile of one pass) to the others
 //                through a descriptor ring in shared memory.  Sub-item j uses K stage j % 5, TMEM buffer
@@ -52,7 +53,6 @@ constexpr int kMma2Warp = 3 + kConsumerWarps;
 constexpr int kThreads = 32 * (4 + kConsumerWarps);
 constexpr uint32_t kHalfBytes = 128 * 128;          // 128 rows x 64 bf16
 constexpr uint32_t kTileBytes = 2 * kHalfBytes;     // 128 rows x 128 bf16
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 constexpr float kMinRowMax = -1.0e30f;              // stands in for "no visible key yet"
 
 // x = (q.k) * log2(e) / sqrt(128)
@@ -89,19 +89,8 @@ struct TcArgs {
   int* ready;           // [C]
   int* queue;           // [2] next P1 run and next P2 run to hand out
   int* status;
+  unsigned long long wait_ns;   // time limit of every wait
 };
-
-// Optional event trace of one CTA (a profiling build defines CKV_TC_TRACE).
-#ifdef CKV_TC_TRACE
-__device__ long long g_tc_trace[6][1024];
-__device__ unsigned long long g_tc_count[8];  // slots, P1 tiles, P2 tiles, no-ops: not ready / pairing / other
-#define TC_TRACE(ev, jj) \
-  do { if (blockIdx.x == 5 && (jj) < 1024) g_tc_trace[ev][jj] = clock64(); } while (0)
-#define TC_COUNT(i) atomicAdd(&g_tc_count[i], 1ull)
-#else
-#define TC_TRACE(ev, jj) do {} while (0)
-#define TC_COUNT(i) do {} while (0)
-#endif
 
 // What the producer tells the other warps about sub-item j (ring slot j % kRing).
 enum : int { kP1 = 0, kP2 = 1, kNop = 2, kStop = 3 };
@@ -150,7 +139,7 @@ __device__ __forceinline__ unsigned long long global_ns() {
 // Bounded wait on an mbarrier phase.  Returns false after the time limit (or when another warp of
 // the CTA already gave up), having recorded the failure.
 __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
-                                            int code) {
+                                            int code, unsigned long long limit_ns) {
   const unsigned long long t0 = global_ns();
   for (int it = 0;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -159,7 +148,7 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volat
         atomicCAS(status + 1 + (code & 7), 0, code);  // which wait each role was in when the CTA gave up
         return false;
       }
-      if (global_ns() - t0 > kWaitLimitNs) {
+      if (global_ns() - t0 > limit_ns) {
         *abort_flag = 1;
         atomicCAS(status, 0, code);
         return false;
@@ -168,10 +157,10 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volat
   }
 }
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
-                                          int code) {
+                                          int code, unsigned long long limit_ns) {
   for (int it = 0; it < 64; ++it)
     if (mbar_try_wait(bar, parity)) return true;
-  return mbar_wait_slow(bar, parity, abort_flag, status, code);
+  return mbar_wait_slow(bar, parity, abort_flag, status, code, limit_ns);
 }
 
 __device__ __forceinline__ void tma_load_5d(const CUtensorMap* map, uint32_t dst, uint32_t bar, int c0, int c1, int c2,
@@ -364,24 +353,6 @@ __device__ __forceinline__ float2 merge_pairs(const float2* p, int count) {
   return make_float2(m, l);
 }
 
-// Bounded wait on a flag in shared memory written by another warp of the CTA.
-template <typename Pred>
-__device__ __forceinline__ bool wait_flag(Pred pred, unsigned sleep_ns, volatile int* abort_flag, int* status, int code) {
-  const unsigned long long t0 = global_ns();
-  for (int it = 1; !pred(); ++it) {
-    __nanosleep(sleep_ns);
-    if ((it & 63) == 0) {
-      if (*abort_flag) return false;
-      if (global_ns() - t0 > kWaitLimitNs) {
-        *abort_flag = 1;
-        atomicCAS(status, 0, code);
-        return false;
-      }
-    }
-  }
-  return true;
-}
-
 // kGrouped: pass 2 writes the per-group maximum and mass (TcArgs::zgrp) instead of per-head column sums.
 template <int W, bool kGrouped>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -464,7 +435,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           // j - kStages; a younger reader needs its own stage's barrier.
           if (ln.q_last > j - kStages)
             ok = mbar_wait(smem_u32(&sm.empty[ln.q_last % kStages]), (ln.q_last / kStages) & 1, abort_flag, a.status,
-                           12 | (j << 8));
+                           12 | (j << 8), a.wait_ns);
           if (!ok) return;
           ++ln.q_loads;
           ln.q_chunk = ln.chunk;
@@ -491,7 +462,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         }
         tma_load_5d(&k_map, smem_u32(sm.k[stage]), bar, 0, tile * kTile, 0, ln.g, ln.u,
                     ln.type == kP1 ? pol_k0 : pol_k1);
-        TC_TRACE(1, j);
         if (++ln.k == ln.tr && ln.type == kP2) {
           // the run's biases may be replaced once its readers are done: tell the scout where it ended
           *(volatile int*)&sm.gen_last_j[ln.gen % kBiasBufs] = j;
@@ -507,16 +477,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           Lane& ln = slot == 0 ? ln0 : ln1;
           if (ln.k == ln.tr) refill(ln, slot == 1);
           ok = ok && mbar_wait(smem_u32(&sm.empty[j % kStages]), ((j / kStages) & 1) ^ 1, abort_flag, a.status,
-                               11 | (j << 8));
-          TC_TRACE(0, j);
+                               11 | (j << 8), a.wait_ns);
           if (!ok) break;
-          TC_COUNT(0);
           *(volatile int*)&sm.prod_j = j;
           if (ln.k < ln.tr) {
-            TC_COUNT(1 + ln.type);
             issue(ln, slot);
           } else {
-            TC_COUNT(3);
             ++idle;
             sm.desc[j % kRing].type = kNop;
             mbar_arrive(smem_u32(&sm.full[j % kFullBars]));
@@ -527,7 +493,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           __nanosleep(200);
           if (*abort_flag) {
             ok = false;
-          } else if (global_ns() - t_busy > kWaitLimitNs) {
+          } else if (global_ns() - t_busy > a.wait_ns) {
             *abort_flag = 1;
             atomicCAS(a.status, 0, 16 | (j << 8));
             ok = false;
@@ -538,7 +504,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       }
       // one stop marker per consumer group
       for (int e = 0; e < kTmemBufs && ok; ++e, ++j) {
-        ok = mbar_wait(smem_u32(&sm.empty[j % kStages]), ((j / kStages) & 1) ^ 1, abort_flag, a.status, 14 | (j << 8));
+        ok = mbar_wait(smem_u32(&sm.empty[j % kStages]), ((j / kStages) & 1) ^ 1, abort_flag, a.status, 14 | (j << 8), a.wait_ns);
         if (ok) {
           sm.desc[j % kRing].type = kStop;
           mbar_arrive(smem_u32(&sm.full[j % kFullBars]));
@@ -613,7 +579,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         __nanosleep(100);
         if ((++it & 63) == 0) {
           bool give_up = *abort_flag != 0;
-          if (!give_up && global_ns() - t_progress > kWaitLimitNs) {
+          if (!give_up && global_ns() - t_progress > a.wait_ns) {
             give_up = true;
             if (lane == 0) *abort_flag = 1, atomicCAS(a.status, 0, 13 | (G << 8));
           }
@@ -632,15 +598,14 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       int stops = 0;
       for (int j = warp == 1 ? 0 : 1; ok && stops < kTmemBufs / 2; j += 2) {
         const int stage = j % kStages, buf = j % kTmemBufs;
-        ok = mbar_wait(smem_u32(&sm.full[j % kFullBars]), (j / kFullBars) & 1, abort_flag, a.status, 21 | (j << 8));
-        TC_TRACE(2, j);
+        ok = mbar_wait(smem_u32(&sm.full[j % kFullBars]), (j / kFullBars) & 1, abort_flag, a.status, 21 | (j << 8), a.wait_ns);
         if (!ok) break;
         const int tq = sm.desc[j % kRing].type;
         const int type = tq & 0xff;
-        ok = mbar_wait(smem_u32(&sm.tmem_empty[buf]), ((j / kTmemBufs) & 1) ^ 1, abort_flag, a.status, 22 | (j << 8));
+        ok = mbar_wait(smem_u32(&sm.tmem_empty[buf]), ((j / kTmemBufs) & 1) ^ 1, abort_flag, a.status, 22 | (j << 8), a.wait_ns);
         if (!ok) break;
         if (type == kP1 || type == kP2) {
-          ok = mbar_wait(smem_u32(&sm.q_full[j & 1]), (tq >> 9) & 1, abort_flag, a.status, 23 | (j << 8));
+          ok = mbar_wait(smem_u32(&sm.q_full[j & 1]), (tq >> 9) & 1, abort_flag, a.status, 23 | (j << 8), a.wait_ns);
           if (!ok) break;
           tc_fence_after();
           const uint32_t kd = k_lo + stage * (kTileBytes >> 4);
@@ -654,7 +619,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           }
           umma_commit(smem_u32(&sm.empty[stage]));
           umma_commit(smem_u32(&sm.tmem_full[buf]));
-          TC_TRACE(3, j);
         } else {
           stops += type == kStop;
           mbar_arrive(smem_u32(&sm.empty[stage]));
@@ -670,9 +634,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     const uint32_t bar_full = smem_u32(&sm.tmem_full[group]), bar_empty = smem_u32(&sm.tmem_empty[group]);
     float m_run = kMinRowMax, l_run = 0.f;
     for (int j = group;; j += kTmemBufs) {
-      bool ok = mbar_wait(bar_full, (j / kTmemBufs) & 1, abort_flag, a.status, 31 | (j << 8));
+      bool ok = mbar_wait(bar_full, (j / kTmemBufs) & 1, abort_flag, a.status, 31 | (j << 8), a.wait_ns);
       ok = __all_sync(0xffffffffu, ok);
-      if (quad == 0 && lane == 0) TC_TRACE(4, j);
       if (!ok) break;
       Desc d = sm.desc[j % kRing];
       d.type &= 0xff;
@@ -855,7 +818,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           a.mgrp[o] = msum;
         }
       }
-      if (quad == 0 && lane == 0) TC_TRACE(5, j);
     }
   }
 
@@ -924,17 +886,6 @@ cudaError_t launch_w(const CUtensorMap& qm, const CUtensorMap& km, const TcArgs&
 
 }  // namespace
 
-#ifdef CKV_TC_TRACE
-extern "C" __attribute__((visibility("default"))) int ckv_debug_tc_counts(unsigned long long* out, int reset) {
-  if (cudaMemcpyFromSymbol(out, g_tc_count, sizeof(g_tc_count)) != cudaSuccess) return 1;
-  unsigned long long z[8] = {};
-  return reset && cudaMemcpyToSymbol(g_tc_count, z, sizeof(z)) != cudaSuccess;
-}
-extern "C" __attribute__((visibility("default"))) int ckv_debug_tc_trace(long long* out) {
-  return cudaMemcpyFromSymbol(out, g_tc_trace, sizeof(long long) * 6 * 1024) != cudaSuccess;
-}
-#endif
-
 bool score_tc_supported(const ckv_shape& s) {
   if (s.dtype != CKV_BF16) return false;
   if (s.window != 16 && s.window != 32 && s.window != 64) return false;
@@ -996,6 +947,7 @@ cudaError_t launch_score_tc(const ckv_shape& s, const void* q, const void* k, fl
   a.q_split = hpb_box * a.W < kTile;  // a short box would pack its halves closer than the operand layout wants
   a.csum = csum, a.part = (float2*)part, a.stat = (float2*)stat;
   a.done = flags, a.ready = flags + 4 * a.C, a.queue = flags + 5 * a.C, a.status = status;
+  a.wait_ns = wait_limit_ns();
   CUtensorMap qm, km;
   {
     // Q: [unit][half][head][row][64]; box = one row block (hpb heads x W rows) x both halves

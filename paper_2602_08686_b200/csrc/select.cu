@@ -17,6 +17,7 @@
 #include <cooperative_groups.h>
 
 #include <algorithm>
+#include <atomic>
 
 #include "ckv_common.cuh"
 
@@ -90,8 +91,8 @@ __device__ __forceinline__ bool barrier_test(uint64_t* bar, uint32_t parity) {
       : "memory");
   return done != 0;
 }
-// Waits for the phase with the given parity, for two seconds at most.
-__device__ __forceinline__ bool barrier_wait_bounded(uint64_t* bar, uint32_t parity) {
+// Waits for the phase with the given parity, for limit_ns at most.
+__device__ __forceinline__ bool barrier_wait_bounded(uint64_t* bar, uint32_t parity, unsigned long long limit_ns) {
   if (barrier_test(bar, parity)) return true;
   unsigned long long t0, t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
@@ -100,7 +101,7 @@ __device__ __forceinline__ bool barrier_wait_bounded(uint64_t* bar, uint32_t par
     for (int i = 0; i < 64; ++i)
       if (barrier_test(bar, parity)) return true;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    if (t - t0 > 2000000000ull) return false;
+    if (t - t0 > limit_ns) return false;
   }
 }
 constexpr int kSelectTimeoutCode = 51;   // status word: a cluster exchange of the selection gave up
@@ -113,7 +114,8 @@ __global__ void __launch_bounds__(kThreads) select_sliced_kernel(ckv_shape s, in
                                                                  const float* __restrict__ scores,
                                                                  const int32_t* __restrict__ budgets,
                                                                  const int32_t* __restrict__ offsets,
-                                                                 int32_t* __restrict__ indices, int* __restrict__ status) {
+                                                                 int32_t* __restrict__ indices, int* __restrict__ status,
+                                                                 unsigned long long wait_ns) {
   extern __shared__ __align__(16) uint32_t stage[];   // [warps in use][1024] score bits in position order
   __shared__ __align__(8) uint2 wcnt[2][kCluster][kWarps];
   __shared__ uint32_t wtot[kWarps];
@@ -220,7 +222,7 @@ __global__ void __launch_bounds__(kThreads) select_sliced_kernel(ckv_shape s, in
         if (lane < kCluster)
           store_credit(cluster_address(&wcnt[st & 1][rank][warp], lane), (uint64_t)r1 | ((uint64_t)r2 << 32),
                        cluster_address(bar, lane));
-        if (warp == 0 && !barrier_wait_bounded(bar, (phase >> (st & 1)) & 1u) && lane == 0) {
+        if (warp == 0 && !barrier_wait_bounded(bar, (phase >> (st & 1)) & 1u, wait_ns) && lane == 0) {
           dead_s = 1;
           atomicCAS(status, 0, kSelectTimeoutCode);
         }
@@ -453,10 +455,14 @@ cudaError_t launch_sliced(const ckv_shape& s, int n, int64_t unit_rows, const fl
   attr[1] = pdl_attribute();
   cfg.attrs = attr, cfg.numAttrs = 2;
   // as many CTAs (clusters) as the device holds at once; each loops over its share of the heads
-  static int resident = 0;   // one CTA of this kernel fills an SM: the answer depends on the device only
+  // one CTA of this kernel fills an SM: the answer depends on the device only, and is remembered per device
+  static std::atomic<int> resident_of[kMaxDevices];
+  int dev = 0;
+  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  int resident = resident_of[dev].load(std::memory_order_relaxed);
   if (resident == 0) {
-    int dev = 0, sms = 0, clusters = 0;
-    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    int sms = 0, clusters = 0;
     if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
     clusters = sms / kCluster;
     if (kCluster > 1) {
@@ -468,10 +474,12 @@ cudaError_t launch_sliced(const ckv_shape& s, int n, int64_t unit_rows, const fl
         (void)cudaGetLastError();
     }
     resident = clusters > 0 ? clusters : 1;
+    resident_of[dev].store(resident, std::memory_order_relaxed);
   }
   const int n_heads = s.n_units * s.n_kv_heads;
   cfg.gridDim = dim3((unsigned)(std::min(n_heads, resident) * kCluster));
-  return cudaLaunchKernelEx(&cfg, select_sliced_kernel<kCluster>, s, unit_rows, scores, budgets, offsets, indices, status);
+  return cudaLaunchKernelEx(&cfg, select_sliced_kernel<kCluster>, s, unit_rows, scores, budgets, offsets, indices, status,
+                            wait_limit_ns());
 }
 
 }  // namespace

@@ -9,8 +9,8 @@ import torch
 
 import oracle
 from paper_2602_08686_b200 import inputs as gen
-from test_gpu_parity import (SCORE_RTOL, check_bucket, check_selection_against_oracle, check_structure, params_of,
-                             problem_of)
+from test_gpu_parity import (SCORE_RTOL, Guarded, check_bucket, check_selection_against_oracle, check_structure,
+                             compress_guarded, params_of, problem_of)
 
 pytestmark = pytest.mark.gpu
 
@@ -57,7 +57,7 @@ def run_full(B, cfg, units, sample, census=True):
     b = gen.make_batch(cfg, "cuda", units)
     Nu = len(units)
     prob = problem_of(cfg, Nu)
-    out = B.compress(b["q"], b["k"], b["v"], b["head_w"], b["sens"], params_of(B, prob), want_scores=True)
+    out = compress_guarded(B, b, params_of(B, prob), Guarded())   # outputs and work space between canary bands
     assert B.ckv_device_status(out["ws"]) == B.OK
     idx, bud, off = (out[x].cpu().numpy() for x in ("indices", "budgets", "offsets"))
     check_structure(idx, bud, off, prob)

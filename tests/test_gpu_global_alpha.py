@@ -89,3 +89,91 @@ def test_staged_calls_with_the_exchange_step(B):
         B.ckv_global_scores(shape, params, hw, total, 8, scores, colmass)
         ref = whole["scores"][4 * r: 4 * r + 4]
         assert torch.allclose(scores, ref, rtol=2e-6, atol=0), (scores - ref).abs().max()
+
+
+def test_gate_table_20_by_4_with_prompt_global_risk(B):
+    """The paper's full gate (Sec. 4.3, Alg. 1 (D)): tau = T_gate[l, b_ent, b_ppl, B_l] on a 20 x 4 entropy x
+    perplexity grid, one table row per layer, the perplexity bin supplied per prompt and repeated for its units, the
+    entropy bin computed from the prompt-global window mass.  Two prompts of three layers; the table was compiled
+    for 32 layers and is mapped to the model's depth on the host first."""
+    layers, upp, n_ent, n_ppl, n_bud = 6, 3, 20, 4, 2
+    cfg = gen.shrink(gen.CONFIGS["c2"], n_layers=layers, batch=1, seq_len=3000, budget_per_head=128, n_needles=4,
+                     n_buckets=n_ent)
+    b = gen.make_batch(cfg, "cpu")
+    rng = np.random.default_rng(9)
+    # thresholds around the mean utility (the paper's range is [0.8, 1.0]); every cell different
+    compiled = (0.8 + 0.4 * rng.permutation(32 * n_ent * n_ppl * n_bud) / (32 * n_ent * n_ppl * n_bud)).astype(np.float32)
+    compiled = compiled.reshape(32, n_ent, n_ppl, n_bud)
+    table = B.ckv_gate_depth_map_host(torch.from_numpy(compiled), upp)           # [3, 20, 4, 2]
+    np.testing.assert_allclose(table.numpy(), oracle.depth_map(compiled, upp), rtol=1e-6)
+    ppl_bin = [1, 3]                                                             # per prompt (the caller's)
+    coords = np.array([(u % upp, ppl_bin[u // upp], u % n_bud) for u in range(layers)], np.int32)
+    prob = problem_of(cfg, layers, global_alpha=True, units_per_prompt=upp, gate_layers=upp, ppl_bins=n_ppl,
+                      budget_levels=n_bud, gate_coords=coords)
+    qn, kn, vn, hw = (gen.as_numpy(b[x]) for x in ("q", "k", "v", "head_w"))
+    sc, cm = oracle.score(prob, qn, kn, hw)
+    P = mode_params(B, prob)
+    P.n_gate_layers, P.n_ppl_bins, P.n_budget_levels = upp, n_ppl, n_bud
+    for override in (-1, 0, 7, 19):
+        prob.bucket_override = P.bucket_override = override
+        out = B.compress(*(b[x].cuda() for x in ("q", "k", "v", "head_w")), table.cuda(), P, want_scores=True,
+                         gate_coords=torch.from_numpy(coords).cuda())
+        assert B.ckv_device_status(out["ws"]) == B.OK
+        gs = out["scores"].double().cpu().numpy()
+        assert (np.abs(gs - sc) / np.maximum(np.abs(sc), 1e-20)).max() <= SCORE_RTOL
+        ref = oracle.budget(prob, sc, cm, table.numpy())
+        gpu_bucket = out["bucket"].cpu().numpy()
+        if override >= 0:
+            assert (gpu_bucket == override).all()
+        bud, off, idx = (out[x].cpu().numpy() for x in ("budgets", "offsets", "indices"))
+        # the oracle's budget step on the GPU's own scores with the GPU's entropy bin: exact
+        for u in range(layers):
+            prob_u = problem_of(cfg, 1, bucket_override=int(gpu_bucket[u]), gate_layers=upp, ppl_bins=n_ppl,
+                                budget_levels=n_bud, gate_coords=coords[u:u + 1])
+            mine = oracle.budget(prob_u, gs[u:u + 1], cm[u:u + 1], table.numpy())
+            assert mine["tau"][0] == float(table[coords[u, 0], gpu_bucket[u], coords[u, 1], coords[u, 2]])
+            assert (mine["budgets"][0] == bud[u]).all(), (override, u)
+        assert (gpu_bucket == ref["bucket"]).all() or override < 0
+        np.testing.assert_array_equal(idx, oracle.select(prob, gs, bud, off))
+    # the coordinates matter: another perplexity bin gives other budgets somewhere
+    other = coords.copy()
+    other[:, 1] = (other[:, 1] + 1) % n_ppl
+    out2 = B.compress(*(b[x].cuda() for x in ("q", "k", "v", "head_w")), table.cuda(), P, want_scores=True,
+                      gate_coords=torch.from_numpy(other).cuda())
+    assert not torch.equal(out2["budgets"], out["budgets"])
+
+
+def test_gate_table_through_the_staged_and_the_host_entry_points(B):
+    """ckv_budget with the four-axis table equals the fused call, and ckv_compress_host stages table and coordinates."""
+    layers, n_ent, n_ppl, n_bud = 4, 20, 4, 3
+    cfg = gen.shrink(gen.CONFIGS["c2"], n_layers=layers, batch=1, seq_len=2100, budget_per_head=96, n_needles=4,
+                     n_buckets=n_ent)
+    b = gen.make_batch(cfg, "cuda")
+    g = torch.Generator().manual_seed(5)
+    table = (0.8 + 0.4 * torch.rand(layers, n_ent, n_ppl, n_bud, generator=g)).cuda()
+    coords = torch.tensor([(u, (2 * u + 1) % n_ppl, u % n_bud) for u in range(layers)], dtype=torch.int32)
+    P = B.Params(pool_kind=cfg.pool_kind, pool_size=cfg.pool_size, budget_per_head=cfg.budget_per_head,
+                 floor_per_head=1, n_buckets=n_ent, n_gate_layers=layers, n_ppl_bins=n_ppl, n_budget_levels=n_bud)
+    fused = B.compress(b["q"], b["k"], b["v"], b["head_w"], table, P, want_scores=True, gate_coords=coords.cuda())
+    shape = B.make_shape(b["q"], b["k"])
+    params = B.make_params(P, b["head_w"], table, gate_coords=coords.cuda())
+    ws = B.alloc_workspace(shape, params, "cuda")
+    scores = torch.empty_like(fused["scores"])
+    colmass = torch.empty(layers, cfg.seq_len, device="cuda")
+    B.ckv_score(shape, params, b["q"], b["k"], b["head_w"], scores, colmass, ws)
+    budgets, offsets = torch.zeros_like(fused["budgets"]), torch.zeros_like(fused["offsets"])
+    bucket, entropy = torch.zeros_like(fused["bucket"]), torch.zeros_like(fused["entropy"])
+    B.ckv_budget(shape, params, scores, colmass, table, budgets, offsets, bucket, entropy, ws)
+    for key, val in (("bucket", bucket), ("budgets", budgets), ("offsets", offsets)):
+        assert torch.equal(fused[key], val), key
+    # host entry point: pinned host tensors, host coordinates
+    hp = B.make_params(P, b["head_w"].cpu(), table.cpu(), gate_coords=coords)
+    host = {x: b[x].cpu().pin_memory() for x in ("q", "k", "v", "head_w")}
+    hko, hvo = fused["k_out"].cpu().zero_().pin_memory(), fused["v_out"].cpu().zero_().pin_memory()
+    hidx = fused["indices"].cpu().zero_().pin_memory()
+    hbud, hoff = fused["budgets"].cpu().zero_().pin_memory(), fused["offsets"].cpu().zero_().pin_memory()
+    staging = torch.empty(B.ckv_staging_bytes(shape, hp), dtype=torch.uint8, device="cuda")
+    B.ckv_compress_host(shape, hp, host["q"], host["k"], host["v"], host["head_w"], table.cpu().pin_memory(), hko, hvo,
+                        hidx, hbud, hoff, staging, ws)
+    assert torch.equal(hidx, fused["indices"].cpu()) and torch.equal(hbud, fused["budgets"].cpu())
+    assert torch.equal(hko, fused["k_out"].cpu()) and torch.equal(hvo, fused["v_out"].cpu())

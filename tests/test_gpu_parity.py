@@ -43,6 +43,51 @@ def score_path(request, B):
     B.ckv_set_score_path(prev)
 
 
+class Guarded:
+    """Device tensors with 256 bytes of a canary pattern on either side (in place of a memory checker): a kernel
+    that writes before or past one of its outputs, or outside its work space, changes a canary byte."""
+    CANARY = 0xA5
+
+    def __init__(self):
+        self.items = []
+
+    def new(self, shape, dtype, fill=None, device="cuda"):
+        shape = tuple(int(x) for x in shape)
+        nbytes = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+        raw = torch.full((256 + (nbytes + 255) // 256 * 256 + 256,), self.CANARY, dtype=torch.uint8, device=device)
+        body = raw[256:256 + nbytes].view(dtype).view(shape)
+        if fill is not None:
+            body.fill_(fill)
+        self.items.append((raw, nbytes))
+        return body
+
+    def check(self):
+        torch.cuda.synchronize()
+        for raw, nbytes in self.items:
+            assert bool((raw[:256] == self.CANARY).all()), "write before a buffer"
+            assert bool((raw[256 + nbytes:] == self.CANARY).all()), "write past a buffer"
+
+
+def compress_guarded(B, b, P, guard, ws=None, gate_coords=None):
+    """The fused call with every output and the work space between canary bands; the dict of binding.compress."""
+    shape = B.make_shape(b["q"], b["k"])
+    params = B.make_params(P, b["head_w"], b["sens"], gate_coords=gate_coords)
+    Nu, Hkv, L, W = shape.n_units, shape.n_kv_heads, shape.seq_len, shape.window
+    rows = B.rows_per_unit(shape, params)
+    if ws is None:
+        ws = guard.new((B.ckv_workspace_bytes(shape, params),), torch.uint8)
+    out = dict(k_out=guard.new((Nu, rows, shape.head_dim), b["k"].dtype, 0), v_out=guard.new((Nu, rows, shape.head_dim), b["v"].dtype, 0),
+               indices=guard.new((Nu, rows), torch.int32, -1), budgets=guard.new((Nu, Hkv), torch.int32, 0),
+               offsets=guard.new((Nu, Hkv + 1), torch.int32, 0), bucket=guard.new((Nu,), torch.int32, 0),
+               entropy=guard.new((Nu,), torch.float32, float("nan")),
+               scores=guard.new((Nu, Hkv, L - W), torch.float32, float("nan")), ws=ws)
+    B.ckv_compress(shape, params, b["q"], b["k"], b["v"], b["head_w"], b["sens"], out["k_out"], out["v_out"],
+                   out["indices"], out["budgets"], out["offsets"], ws, scores=out["scores"], bucket=out["bucket"],
+                   entropy=out["entropy"])
+    guard.check()
+    return out
+
+
 def problem_of(cfg, Nu, **kw):
     prob = Problem(Nu, cfg.n_q_heads, cfg.n_kv_heads, cfg.seq_len, cfg.window, head_dim=cfg.head_dim,
                    dtype=oracle.BF16 if cfg.dtype == "bf16" else oracle.F32, pool_kind=cfg.pool_kind,
@@ -137,20 +182,22 @@ def run_case(B, cfg, units=None, **prob_kw):
     P = params_of(B, prob)
     shape = B.make_shape(b["q"], b["k"])
     params = B.make_params(P, b["head_w"], b["sens"])
-    ws = B.alloc_workspace(shape, params, "cuda")
+    guard = Guarded()   # every output and the work space sit between canary bands
+    ws = guard.new((B.ckv_workspace_bytes(shape, params),), torch.uint8)
     n, Hkv, L = prob.n, prob.n_kv_heads, prob.seq_len
     rows = B.rows_per_unit(shape, params)
     dev = "cuda"
 
     # ---- staged path -------------------------------------------------------------------------
-    scores = torch.full((Nu, Hkv, n), float("nan"), device=dev)
-    colmass = torch.full((Nu, L), float("nan"), device=dev)
+    scores = guard.new((Nu, Hkv, n), torch.float32, float("nan"))
+    colmass = guard.new((Nu, L), torch.float32, float("nan"))
     B.ckv_score(shape, params, b["q"], b["k"], b["head_w"], scores, colmass, ws)
-    budgets = torch.zeros(Nu, Hkv, dtype=torch.int32, device=dev)
-    offsets = torch.zeros(Nu, Hkv + 1, dtype=torch.int32, device=dev)
-    bucket = torch.zeros(Nu, dtype=torch.int32, device=dev)
-    entropy = torch.zeros(Nu, device=dev)
+    budgets = guard.new((Nu, Hkv), torch.int32, 0)
+    offsets = guard.new((Nu, Hkv + 1), torch.int32, 0)
+    bucket = guard.new((Nu,), torch.int32, 0)
+    entropy = guard.new((Nu,), torch.float32, 0)
     B.ckv_budget(shape, params, scores, colmass, b["sens"], budgets, offsets, bucket, entropy, ws)
+    guard.check()
     err = check_scores(scores, colmass, entropy, ref, prob)
     check_bucket(bucket, ref, prob)
 
@@ -172,7 +219,7 @@ def run_case(B, cfg, units=None, **prob_kw):
     # (4) select on identical bits
     ref_bud = torch.from_numpy(ref["budgets"]).cuda()
     ref_off = torch.from_numpy(ref["offsets"]).cuda()
-    idx_g = torch.full((Nu, rows), -1, dtype=torch.int32, device=dev)
+    idx_g = guard.new((Nu, rows), torch.int32, -1)
     B.ckv_select(shape, params, s32.cuda(), ref_bud, ref_off, idx_g, ws)
     want = oracle.select(prob, s32.double().numpy(), ref["budgets"], ref["offsets"])
     np.testing.assert_array_equal(idx_g.cpu().numpy(), want)
@@ -181,13 +228,14 @@ def run_case(B, cfg, units=None, **prob_kw):
     check_selection_against_oracle(idx_g.cpu().numpy(), ref["budgets"], ref["offsets"], ref, prob)
 
     # (5) gather
-    k_out = torch.zeros(Nu, rows, prob.head_dim, dtype=b["k"].dtype, device=dev)
-    v_out = torch.zeros_like(k_out)
+    k_out = guard.new((Nu, rows, prob.head_dim), b["k"].dtype, 0)
+    v_out = guard.new((Nu, rows, prob.head_dim), b["k"].dtype, 0)
     B.ckv_gather(shape, params, b["k"], b["v"], idx_g, ref_off, k_out, v_out)
+    guard.check()
     check_gather(b_cpu["k"], b_cpu["v"], k_out, v_out, idx_g.cpu().numpy(), ref["offsets"], prob)
 
     # ---- fused path --------------------------------------------------------------------------
-    out = B.compress(b["q"], b["k"], b["v"], b["head_w"], b["sens"], P, want_scores=True, ws=ws)
+    out = compress_guarded(B, b, P, guard, ws=ws)
     assert B.ckv_device_status(ws) == B.OK
     assert torch.equal(out["scores"], scores)                       # deterministic, same kernels
     gs = out["scores"].double().cpu().numpy()

@@ -89,6 +89,24 @@ def test_argument_errors_are_found_on_the_host():
     bad.kv_stride_tok = 130                                                       # rows not 16-byte aligned
     assert score(bad, p) == B.ERR_INVALID_ARG
     assert B.ckv_workspace_bytes(llama_shape(d=64), p) == 0
+    # broadcast views (a zero stride over more than one unit or head) are refused; over an extent of one they are fine
+    for field in ("q_stride_unit", "q_stride_head", "kv_stride_unit", "kv_stride_head"):
+        bad = llama_shape()
+        setattr(bad, field, 0)
+        assert score(bad, p) == B.ERR_INVALID_ARG, field
+    one = llama_shape(Nu=1)
+    one.q_stride_unit = one.kv_stride_unit = 0
+    assert B.ckv_workspace_bytes(one, p) > 0
+    # the four-axis gate table: its sizes must be given, and it is one table for all units
+    coords = C.cast(fake, C.c_void_p)
+    gate = default_params(n_buckets=20)
+    gate.gate_coords, gate.n_gate_layers, gate.n_ppl_bins, gate.n_budget_levels = coords, 32, 4, 3
+    assert B.ckv_workspace_bytes(s, gate) > 0
+    for field, value in (("n_gate_layers", 0), ("n_ppl_bins", 0), ("n_budget_levels", -1), ("sens_stride_unit", 20)):
+        bad_gate = default_params(n_buckets=20)
+        bad_gate.gate_coords, bad_gate.n_gate_layers, bad_gate.n_ppl_bins, bad_gate.n_budget_levels = coords, 32, 4, 3
+        setattr(bad_gate, field, value)
+        assert score(s, bad_gate) == B.ERR_INVALID_ARG, field
     assert lib.ckv_gather(C.byref(s), C.byref(p), None, fake, fake, fake, fake, fake, None) == B.ERR_INVALID_ARG
     assert lib.ckv_compress_host(C.byref(s), C.byref(p), fake, fake, fake, fake, fake, fake, fake, fake, fake, fake,
                                  fake, 16, fake, big, None) == B.ERR_WORKSPACE    # staging too small
@@ -101,6 +119,52 @@ def test_workspace_grows_with_the_problem():
     c = B.ckv_workspace_bytes(llama_shape(L=32768, Nu=4), p)
     assert 0 < a < b < c
     assert B.ckv_staging_bytes(llama_shape(L=4096), p) > 2 * 2 * 8 * 4096 * 128 * 2
+
+
+def test_score_stage_work_space_and_the_fixed_scratch_limit():
+    """ckv_score needs only the leading sections of the work space, and ckv_score_noalloc accepts what fits its
+    fixed scratch by that measure: two units of the Llama shape at 32k do, three do not."""
+    p = default_params()
+    for Nu in (1, 2, 3):
+        s = llama_shape(Nu=Nu)
+        assert 0 < B.ckv_score_workspace_bytes(s, p) < B.ckv_workspace_bytes(s, p)
+    assert B.ckv_score_workspace_bytes(llama_shape(Nu=2), p) <= B.NOALLOC_SCRATCH_BYTES
+    assert B.ckv_score_workspace_bytes(llama_shape(Nu=3), p) > B.NOALLOC_SCRATCH_BYTES
+    fake = C.c_void_p(1 << 20)   # never dereferenced: the call fails the size test first
+    s3 = llama_shape(Nu=3)
+    assert B.lib().ckv_score_noalloc(C.byref(s3), C.byref(p), fake, fake, fake, fake, fake, None) == B.ERR_WORKSPACE
+
+
+def test_depth_map_matches_the_oracle():
+    rng = np.random.default_rng(3)
+    import torch
+    for n_src, n_dst in ((32, 32), (32, 28), (32, 80), (4, 9), (6, 1), (1, 5)):
+        table = rng.uniform(0.8, 1.0, (n_src, 20, 4, 2)).astype(np.float32)
+        got = B.ckv_gate_depth_map_host(torch.from_numpy(table), n_dst).numpy()
+        want = oracle.depth_map(table, n_dst)
+        assert got.shape == want.shape
+        np.testing.assert_allclose(got, want, rtol=1e-6, atol=0)
+        if n_src == n_dst:
+            np.testing.assert_array_equal(got, table)
+        np.testing.assert_array_equal(got[0], table[0])
+    assert B.lib().ckv_gate_depth_map_host(None, 4, 4, 8, None) == 1
+
+
+def test_binding_refuses_values_laid_out_unlike_the_keys():
+    """ckv_shape has one set of strides for k and v: the binding raises when v is another view."""
+    import torch
+    q = torch.zeros(2, 4, 8, 128, dtype=torch.bfloat16)
+    k = torch.zeros(2, 2, 64, 128, dtype=torch.bfloat16)
+    shape = B.make_shape(q, k)
+    B._check_kv(shape, k, "k")
+    B._check_kv(shape, torch.zeros_like(k), "v")
+    padded = torch.zeros(2, 2, 64, 256, dtype=torch.bfloat16)[..., :128]          # other token stride
+    for bad in (padded, torch.zeros(2, 2, 63, 128, dtype=torch.bfloat16), k.float(),
+                torch.zeros(2, 64, 2, 128, dtype=torch.bfloat16).transpose(1, 2)):
+        with pytest.raises(ValueError):
+            B._check_kv(shape, bad, "v")
+    with pytest.raises(ValueError):
+        B._check_dense(padded, "k_out")
 
 
 def test_budget_split_matches_oracle_and_brute_force():
@@ -163,6 +227,22 @@ assert torch.allclose(pm, mass.sum(1), rtol=1e-6), (pm - mass.sum(1)).abs().max(
 dist.barrier(); dist.destroy_process_group()
 print("rank", rank, "ok")
 """
+
+
+def test_bench_starts_its_own_ranks():
+    """`bench.py --gpus 2` outside a launcher starts two ranks itself; with --dry-run they are CPU ranks under gloo
+    whose step is a sleep (rank r sleeps r + 1 ms), so the line must say two GPUs, twice the units and the slower
+    rank's time."""
+    import json
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "5", "--dry-run"],
+                         stdout=subprocess.PIPE, stderr=subprocess.PIPE, env=env, timeout=300)
+    assert res.returncode == 0, res.stderr.decode()[-2000:]
+    lines = [ln for ln in res.stdout.decode().splitlines() if ln.startswith("{")]
+    assert len(lines) == 1, lines
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["config"]["units_total"] == 64 and line["config"]["units_per_gpu"] == 32
+    assert line["ms_per_step"] >= 2.0 and line["scaling"] == "weak"
 
 
 def test_two_rank_sharding_under_gloo(tmp_path):

@@ -16,8 +16,6 @@ import torch
 
 from paper_2602_08686_b200 import inputs as gen
 
-SCORE_RTOL = 1e-3   # the tolerance of the other GPU score tests
-
 
 def _score_both_ways(B, cfg):
     b = gen.make_batch(cfg, "cuda")
@@ -25,7 +23,7 @@ def _score_both_ways(B, cfg):
                  floor_per_head=cfg.floor_per_head, n_buckets=cfg.n_buckets)
     shape = B.make_shape(b["q"], b["k"])
     params = B.make_params(P, b["head_w"], b["sens"])
-    assert B.ckv_workspace_bytes(shape, params) <= B.NOALLOC_SCRATCH_BYTES
+    assert B.ckv_score_workspace_bytes(shape, params) <= B.NOALLOC_SCRATCH_BYTES
     Nu, Hkv, L, n = cfg.n_units, cfg.n_kv_heads, cfg.seq_len, cfg.n
     want_s = torch.full((Nu, Hkv, n), float("nan"), device="cuda")
     want_c = torch.full((Nu, L), float("nan"), device="cuda")
@@ -35,11 +33,10 @@ def _score_both_ways(B, cfg):
     got_s = torch.full_like(want_s, float("nan"))
     got_c = torch.full_like(want_c, float("nan"))
     B.ckv_score_noalloc(shape, params, b["q"], b["k"], b["head_w"], got_s, got_c)
-    torch.cuda.synchronize()
+    assert B.ckv_device_status(None) == B.OK          # the status word inside the fixed scratch
     assert torch.isfinite(got_s).all() and torch.isfinite(got_c).all()
-    rel_s = ((got_s - want_s).abs() / want_s.abs().clamp_min(1e-20)).max().item()
-    rel_c = ((got_c - want_c).abs() / want_c.abs().clamp_min(1e-20)).max().item()
-    assert rel_s <= SCORE_RTOL and rel_c <= SCORE_RTOL, (rel_s, rel_c)
+    # the same kernels on the same inputs, and the scan is deterministic: the same bits, not just the same values
+    assert torch.equal(got_s, want_s) and torch.equal(got_c, want_c)
 
 
 @pytest.mark.gpu
@@ -62,7 +59,7 @@ def test_noalloc_score_refuses_problems_beyond_its_fixed_scratch():
     H, Hkv, W, d, L, Nu = 32, 8, 32, 128, 32768, 32
     shape = B.ckv_shape(Nu, H, Hkv, d, L, W, B.BF16, 0, H * W * d, W * d, d, Hkv * L * d, L * d, d)
     params = B.ckv_params(B.POOL_MAX, 7, 512, 1, 16, -1, H, 0)
-    assert B.ckv_workspace_bytes(shape, params) > B.NOALLOC_SCRATCH_BYTES
+    assert B.ckv_score_workspace_bytes(shape, params) > B.NOALLOC_SCRATCH_BYTES
     fake = C.c_void_p(1 << 20)   # never dereferenced: the call fails validation first
     rc = B.lib().ckv_score_noalloc(C.byref(shape), C.byref(params), fake, fake, fake, fake, fake, None)
     assert rc == B.ERR_WORKSPACE
