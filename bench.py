@@ -460,7 +460,10 @@ def main():
         hko, hvo = pin(k_out), pin(v_out)
         hidx, hbud, hoff = pin(indices), pin(budgets), pin(offsets)
         staging = torch.empty(B.ckv_staging_bytes(shape, params), dtype=torch.uint8, device=dev)
-        h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv, hw, hs))
+        # V is read in place when the pinned buffer is mapped: only the kept rows cross the bus (as many bytes as v_out)
+        v_bytes = hvo.numel() * hvo.element_size() if B.ckv_reads_in_place(hv) and not args.value_norm else \
+            hv.numel() * hv.element_size()
+        h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hw, hs)) + v_bytes
         d2h = sum(t.numel() * t.element_size() for t in (hko, hvo, hidx, hbud, hoff))
         e2e_steps = max(1, min(args.steps, 3))
 
@@ -478,7 +481,9 @@ def main():
         ms_e2e = max_over_ranks(e0.elapsed_time(e1)) / e2e_steps
         e2e = {"value": world * n_units * L / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "steps": e2e_steps,
-               "api": "ckv_compress_host (pinned host tensors)"}
+               "api": "ckv_compress_host (pinned host tensors)",
+               "values": "kept rows read in place from the pinned host buffer" if v_bytes < hv.numel() * hv.element_size()
+               else "copied whole"}
         wl.step()
         torch.cuda.synchronize()
         assert torch.equal(hidx, indices.cpu())

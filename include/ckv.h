@@ -250,8 +250,14 @@ ckv_status ckv_compress(const ckv_shape* shape, const ckv_params* params, const 
  * ckv_compress, copies k_out, v_out, indices, budgets and offsets back, and synchronises the
  * stream before returning.  Host tensors are dense ([Nu,H,W,d], [Nu,Hkv,L,d], head_w [Nu,H] or [H]
  * by head_w_stride_unit, sens likewise); the strides in `shape` are ignored.
+ * V is only gathered (Alg. 1 (D)) unless params->value_norm streams it: when v_host is page-locked memory that the
+ * device has mapped (ckv_reads_in_place(v_host) == 1; true of cudaHostAlloc / cudaHostRegister memory on systems
+ * with unified addressing), V is not copied at all and the gather reads the kept rows from the host buffer in
+ * place, so that of V only Hkv * min(B, L) rows per unit cross the bus.  Pageable memory is copied as a whole.
  */
 size_t ckv_staging_bytes(const ckv_shape* shape, const ckv_params* params);
+/* 1 if a kernel can read this host buffer in place (see ckv_compress_host), 0 if it would be copied. */
+int ckv_reads_in_place(const void* host_pointer);
 ckv_status ckv_compress_host(const ckv_shape* shape, const ckv_params* params, const void* q_win_host,
                              const void* k_host, const void* v_host, const float* head_w_host,
                              const float* sens_host, void* k_out_host, void* v_out_host,

@@ -223,6 +223,12 @@ def ckv_score_workspace_bytes(shape: ckv_shape, params: ckv_params) -> int:
     return int(lib().ckv_score_workspace_bytes(C.byref(shape), C.byref(params)))
 
 
+def ckv_reads_in_place(host_tensor: torch.Tensor) -> bool:
+    """True if ckv_compress_host would read this host tensor in place (page-locked and mapped) instead of copying it."""
+    lib().ckv_reads_in_place.argtypes = [C.c_void_p]
+    return bool(lib().ckv_reads_in_place(_ptr(host_tensor)))
+
+
 def ckv_staging_bytes(shape: ckv_shape, params: ckv_params) -> int:
     return int(lib().ckv_staging_bytes(C.byref(shape), C.byref(params)))
 

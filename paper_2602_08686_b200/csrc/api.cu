@@ -376,6 +376,19 @@ ckv_status ckv_compress(const ckv_shape* shape, const ckv_params* params, const 
   return CKV_OK;
 }
 
+// Device address under which a kernel can read a host buffer in place (page-locked memory that the device has
+// mapped), or null when the buffer has to be copied.
+static const void* mapped_host_pointer(const void* host) {
+  cudaPointerAttributes at{};
+  if (cudaPointerGetAttributes(&at, host) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return nullptr;
+  }
+  return at.type == cudaMemoryTypeHost ? at.devicePointer : nullptr;
+}
+
+int ckv_reads_in_place(const void* host_pointer) { return host_pointer && mapped_host_pointer(host_pointer) ? 1 : 0; }
+
 // staging sections: q | k | v | head_w | sens | k_out | v_out | indices | budgets | offsets
 struct Staging {
   size_t q, k, v, head_w, sens, k_out, v_out, indices, budgets, offsets, total;
@@ -445,14 +458,20 @@ ckv_status ckv_compress_host(const ckv_shape* shape, const ckv_params* params, c
   cudaStream_t st = (cudaStream_t)stream;
   CKV_CUDA(cudaMemcpyAsync(d + g.q, q_win_host, g.q_b, cudaMemcpyHostToDevice, st));
   CKV_CUDA(cudaMemcpyAsync(d + g.k, k_host, g.kv_b, cudaMemcpyHostToDevice, st));
-  CKV_CUDA(cudaMemcpyAsync(d + g.v, v_host, g.kv_b, cudaMemcpyHostToDevice, st));
+  // The values are only gathered (unless the value-norm ratio streams them): where the device can read the host
+  // buffer in place, the gather fetches the kept rows from there and the other 98 % of V never cross the bus.
+  const void* v_dev = params->value_norm ? nullptr : mapped_host_pointer(v_host);
+  if (!v_dev) {
+    CKV_CUDA(cudaMemcpyAsync(d + g.v, v_host, g.kv_b, cudaMemcpyHostToDevice, st));
+    v_dev = d + g.v;
+  }
   CKV_CUDA(cudaMemcpyAsync(d + g.head_w, head_w_host, g.hw_b, cudaMemcpyHostToDevice, st));
   CKV_CUDA(cudaMemcpyAsync(d + g.sens, sens_host, g.sens_b, cudaMemcpyHostToDevice, st));
   if (params->gate_coords) {
     CKV_CUDA(cudaMemcpyAsync(d + g.coords, params->gate_coords, g.coords_b, cudaMemcpyHostToDevice, st));
     p.gate_coords = reinterpret_cast<const int32_t*>(d + g.coords);
   }
-  CKV_TRY(ckv_compress(&s, &p, d + g.q, d + g.k, d + g.v, (const float*)(d + g.head_w), (const float*)(d + g.sens),
+  CKV_TRY(ckv_compress(&s, &p, d + g.q, d + g.k, v_dev, (const float*)(d + g.head_w), (const float*)(d + g.sens),
                        d + g.k_out, d + g.v_out, (int32_t*)(d + g.indices), (int32_t*)(d + g.budgets),
                        (int32_t*)(d + g.offsets), nullptr, nullptr, nullptr, ws, ws_bytes, stream));
   CKV_CUDA(cudaMemcpyAsync(k_out_host, d + g.k_out, g.out_b, cudaMemcpyDeviceToHost, st));

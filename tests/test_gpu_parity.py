@@ -585,10 +585,24 @@ def test_compress_host_matches_device_path(B):
     off = pin(torch.zeros(2, 3, dtype=torch.int32))
     staging = torch.empty(B.ckv_staging_bytes(shape, params), dtype=torch.uint8, device="cuda")
     ws = B.alloc_workspace(shape, params, "cuda")
-    B.ckv_compress_host(shape, params, pin(b["q"]), pin(b["k"]), pin(b["v"]), pin(b["head_w"]), pin(b["sens"]),
-                        k_out, v_out, idx, bud, off, staging, ws)
-    assert torch.equal(idx, dev["indices"].cpu()) and torch.equal(bud, dev["budgets"].cpu())
-    assert torch.equal(k_out, dev["k_out"].cpu()) and torch.equal(v_out, dev["v_out"].cpu())
+    # page-locked values are read in place by the gather (only the kept rows cross the bus); pageable ones are copied;
+    # with the value-norm ratio the values are streamed on the device, hence copied as well: same results every way
+    v_pinned = pin(b["v"])
+    assert B.ckv_reads_in_place(v_pinned) and not B.ckv_reads_in_place(b["v"])
+    for v_host in (v_pinned, b["v"]):
+        for t in (k_out, v_out, idx, bud, off):
+            t.zero_()
+        B.ckv_compress_host(shape, params, pin(b["q"]), pin(b["k"]), v_host, pin(b["head_w"]), pin(b["sens"]),
+                            k_out, v_out, idx, bud, off, staging, ws)
+        assert torch.equal(idx, dev["indices"].cpu()) and torch.equal(bud, dev["budgets"].cpu())
+        assert torch.equal(k_out, dev["k_out"].cpu()) and torch.equal(v_out, dev["v_out"].cpu())
+    P.value_norm = True
+    dev_vn = B.compress(*(b[x].cuda() for x in ("q", "k", "v", "head_w", "sens")), P)
+    params_vn = B.make_params(P, b["head_w"], b["sens"])
+    ws_vn = B.alloc_workspace(shape, params_vn, "cuda")
+    B.ckv_compress_host(shape, params_vn, pin(b["q"]), pin(b["k"]), v_pinned, pin(b["head_w"]), pin(b["sens"]),
+                        k_out, v_out, idx, bud, off, staging, ws_vn)
+    assert torch.equal(idx, dev_vn["indices"].cpu()) and torch.equal(v_out, dev_vn["v_out"].cpu())
 
 
 def test_deterministic_run_to_run(B):
