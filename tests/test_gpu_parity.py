@@ -22,7 +22,7 @@ from paper_2602_08686_b200 import inputs as gen
 
 pytestmark = pytest.mark.gpu
 
-SCORE_RTOL = 1e-3          # spec tolerance on pooled, weighted scores
+SCORE_RTOL = 1e-3          # tolerance on pooled, weighted scores (max relative error)
 TIE_BAND = 1e-3            # selection may differ only inside this relative band around the k-th score
 
 
