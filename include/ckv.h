@@ -14,10 +14,11 @@
  *   - The caller owns every buffer.  The library allocates no device memory and
  *     keeps no per-call state; work space is passed in (`ws`, `ws_bytes`, at
  *     least ckv_workspace_bytes(), 256-byte aligned).  What the library does keep,
- *     per process: the diagnostic settings of ckv_set_score_path and ckv_set_tunable
- *     (results do not depend on them), a launch counter, and per-device constants it
- *     looks up once (driver entry point, resident CTAs, the address of the fixed scratch);
- *     per calling thread: the event pair of ckv_set_scan_events.
+ *     per process: the defaults of the scheduling settings (ckv_set_score_path,
+ *     ckv_set_tunable; results do not depend on them, and a call can carry its own in
+ *     params->tuning), a launch counter, and per-device constants it looks up once
+ *     (driver entry point, resident CTAs, the address of the fixed scratch); per calling
+ *     thread: the default event pair of ckv_set_scan_events.
  *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL is
  *     the default stream) and return after the last launch was queued.
  *   - Errors are return codes.  Argument errors are found on the host before
@@ -67,6 +68,21 @@ typedef struct {
   int64_t kv_stride_unit, kv_stride_head, kv_stride_tok; /* elements; shared by k and v */
 } ckv_shape;
 
+/* Optional per-call settings of how the work is scheduled (never of what is computed: the results do not depend
+ * on them).  A field of -1 (a null event) takes the process-wide default that ckv_set_score_path / ckv_set_tunable
+ * (for the events: the calling thread's ckv_set_scan_events pair) last set.  Calls on different threads or streams
+ * may carry different settings. */
+typedef struct {
+  int32_t score_path;   /* -1, or as ckv_set_score_path: 0 automatic, 1 plain kernels, 2 tensor-core kernel required */
+  int32_t run_tiles;    /* -1, or 1..64 */
+  int32_t l2_hints;     /* -1, 0, 1 */
+  int32_t group_fuse;   /* -1, 0, 1 */
+  int32_t pdl;          /* -1, 0, 1 */
+  int32_t reserved_;    /* set to 0 */
+  void* scan_start_event;   /* cudaEvent_t pair recorded around the tensor-core scan of this call, or NULL */
+  void* scan_stop_event;
+} ckv_tuning;
+
 typedef struct {
   int32_t pool_kind;        /* ckv_pool */
   int32_t pool_size;        /* odd, 1..15; 1 (or CKV_POOL_NONE) is the paper's un-pooled score */
@@ -107,6 +123,7 @@ typedef struct {
   int32_t n_budget_levels;  /* >= 1 with gate_coords */
   int32_t reserved2_;       /* set to 0 */
   const int32_t* gate_coords;
+  const ckv_tuning* tuning; /* HOST pointer read before the call returns, or NULL for the defaults */
 } ckv_params;
 
 /* Bytes of work space any entry point needs for this problem (0 on invalid arguments). */

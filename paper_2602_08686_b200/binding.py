@@ -33,6 +33,23 @@ class ckv_shape(C.Structure):
                                          "kv_stride_unit", "kv_stride_head", "kv_stride_tok")]
 
 
+class ckv_tuning(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("score_path", "run_tiles", "l2_hints", "group_fuse", "pdl", "reserved_")] + \
+               [("scan_start_event", C.c_void_p), ("scan_stop_event", C.c_void_p)]
+
+
+def make_tuning(score_path: int = -1, run_tiles: int = -1, l2_hints: int = -1, group_fuse: int = -1, pdl: int = -1,
+                scan_events=None) -> ckv_tuning:
+    """Per-call scheduling settings (-1: the process-wide default); scan_events is a pair of torch.cuda.Event objects
+    (timing enabled, recorded once before) to be recorded around the tensor-core scan of the calls that carry it."""
+    ev0 = ev1 = None
+    if scan_events is not None:
+        ev0, ev1 = (C.c_void_p(e.cuda_event) for e in scan_events)
+    t = ckv_tuning(score_path, run_tiles, l2_hints, group_fuse, pdl, 0, ev0, ev1)
+    t._keep = scan_events
+    return t
+
+
 class ckv_params(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("pool_kind", "pool_size", "budget_per_head", "floor_per_head",
                                          "n_buckets", "bucket_override")] + \
@@ -40,7 +57,7 @@ class ckv_params(C.Structure):
                [("value_norm", C.c_int32), ("value_norm_eps", C.c_float), ("shared_elastic", C.c_int32),
                 ("global_alpha", C.c_int32), ("units_per_prompt", C.c_int32), ("reserved_", C.c_int32),
                 ("n_gate_layers", C.c_int32), ("n_ppl_bins", C.c_int32), ("n_budget_levels", C.c_int32),
-                ("reserved2_", C.c_int32), ("gate_coords", C.c_void_p)]
+                ("reserved2_", C.c_int32), ("gate_coords", C.c_void_p), ("tuning", C.POINTER(ckv_tuning))]
 
 
 _lib = None
@@ -164,7 +181,7 @@ def make_shape(q: torch.Tensor, k: torch.Tensor) -> ckv_shape:
 
 
 def make_params(p: Params, head_w: torch.Tensor | None, sens: torch.Tensor | None, H: int = 0,
-                gate_coords: torch.Tensor | None = None) -> ckv_params:
+                gate_coords: torch.Tensor | None = None, tuning: ckv_tuning | None = None) -> ckv_params:
     """Parameter struct.  With gate_coords ([Nu,3] int32: layer row, perplexity bin, budget level per unit; on the
     device, or on the host for ckv_compress_host) `sens` is the dense table [n_gate_layers, n_buckets, n_ppl_bins,
     n_budget_levels]; the struct keeps a reference to the tensor."""
@@ -180,8 +197,9 @@ def make_params(p: Params, head_w: torch.Tensor | None, sens: torch.Tensor | Non
                      p.bucket_override, hw_stride, se_stride, int(p.value_norm), float(p.value_norm_eps),
                      int(p.shared_elastic), int(p.global_alpha), int(p.units_per_prompt), 0,
                      int(p.n_gate_layers) if gate_coords is not None else 0, int(p.n_ppl_bins),
-                     int(p.n_budget_levels), 0, None if gate_coords is None else gate_coords.data_ptr())
-    out._keep = gate_coords
+                     int(p.n_budget_levels), 0, None if gate_coords is None else gate_coords.data_ptr(),
+                     None if tuning is None else C.pointer(tuning))
+    out._keep = (gate_coords, tuning)
     return out
 
 
@@ -365,10 +383,10 @@ def ckv_allocate_rows_host(n: int, f: int, P: int, demands) -> list[int]:
 
 # ------------------------------------------------------------------------------------ convenience
 def compress(q_win, k, v, head_w, sens, p: Params, want_scores: bool = False, ws=None, stream=None,
-             gate_coords=None):
+             gate_coords=None, tuning=None):
     """Allocates the outputs and the work space with torch and runs ckv_compress."""
     shape = make_shape(q_win, k)
-    params = make_params(p, head_w, sens, gate_coords=gate_coords)
+    params = make_params(p, head_w, sens, gate_coords=gate_coords, tuning=tuning)
     dev = k.device
     Nu, Hkv = shape.n_units, shape.n_kv_heads
     rows = rows_per_unit(shape, params)

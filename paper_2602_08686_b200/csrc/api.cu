@@ -12,11 +12,42 @@ namespace ckv {
 static std::atomic<int64_t> g_launches{0};
 static std::atomic<int> g_score_path{0};  // 0 = automatic, 1 = plain kernels, 2 = tensor-core kernel
 static std::atomic<int> g_pdl{1};         // 1: the kernels after the pooling kernel use programmatic dependent launch
-bool pdl_enabled() { return g_pdl.load(std::memory_order_relaxed) != 0; }
 static std::atomic<int> g_group_fuse{1};  // 1: the scan writes per-group maxima and masses where it can
+static std::atomic<int> g_run_tiles{16};  // key tiles per run of the tensor-core scan
+static std::atomic<int> g_l2_hints{1};    // 1: first-pass K loads keep their lines in L2, second-pass loads release them
 static std::atomic<unsigned long long> g_wait_limit_ns{2000000000ull};   // bound of every device-side wait
 unsigned long long wait_limit_ns() { return g_wait_limit_ns.load(std::memory_order_relaxed); }
 static thread_local cudaEvent_t t_scan_start = nullptr, t_scan_stop = nullptr;  // see ckv_set_scan_events
+
+// The scheduling settings of one call: params->tuning where it gives a value, the process-wide defaults elsewhere.
+// An entry point resolves them once and makes them current for its thread while it queues its launches, so that the
+// launchers need no extra arguments and concurrent calls on other threads keep their own.
+struct CallTuning {
+  int score_path, run_tiles, l2_hints, group_fuse, pdl;
+  cudaEvent_t ev0, ev1;
+};
+static thread_local const CallTuning* t_call = nullptr;
+static CallTuning resolve_tuning(const ckv_params& p) {
+  const ckv_tuning* t = p.tuning;
+  CallTuning c;
+  c.score_path = t && t->score_path >= 0 ? t->score_path : g_score_path.load(std::memory_order_relaxed);
+  c.run_tiles = t && t->run_tiles >= 0 ? t->run_tiles : g_run_tiles.load(std::memory_order_relaxed);
+  c.l2_hints = t && t->l2_hints >= 0 ? t->l2_hints : g_l2_hints.load(std::memory_order_relaxed);
+  c.group_fuse = t && t->group_fuse >= 0 ? t->group_fuse : g_group_fuse.load(std::memory_order_relaxed);
+  c.pdl = t && t->pdl >= 0 ? t->pdl : g_pdl.load(std::memory_order_relaxed);
+  c.ev0 = t && t->scan_start_event ? (cudaEvent_t)t->scan_start_event : t_scan_start;
+  c.ev1 = t && t->scan_stop_event ? (cudaEvent_t)t->scan_stop_event : t_scan_stop;
+  return c;
+}
+struct TuningScope {
+  CallTuning mine;
+  const CallTuning* outer;
+  explicit TuningScope(const ckv_params& p) : mine(resolve_tuning(p)), outer(t_call) { t_call = &mine; }
+  ~TuningScope() { t_call = outer; }
+};
+bool pdl_enabled() { return (t_call ? t_call->pdl : g_pdl.load(std::memory_order_relaxed)) != 0; }
+int tuning_run_tiles() { return t_call ? t_call->run_tiles : g_run_tiles.load(std::memory_order_relaxed); }
+int tuning_l2_hints() { return t_call ? t_call->l2_hints : g_l2_hints.load(std::memory_order_relaxed); }
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
 static size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
@@ -97,6 +128,11 @@ static ckv_status check_params(const ckv_shape* s, const ckv_params* p) {
   if (p->bucket_override < -1 || p->bucket_override >= p->n_buckets) return CKV_ERR_INVALID_ARG;
   if (p->head_w_stride_unit < 0 || p->sens_stride_unit < 0) return CKV_ERR_INVALID_ARG;
   if (p->value_norm != 0 && p->value_norm != 1) return CKV_ERR_INVALID_ARG;
+  if (const ckv_tuning* t = p->tuning) {
+    if (t->score_path < -1 || t->score_path > 2 || t->run_tiles < -1 || t->run_tiles == 0 || t->run_tiles > 64 ||
+        t->l2_hints < -1 || t->l2_hints > 1 || t->group_fuse < -1 || t->group_fuse > 1 || t->pdl < -1 || t->pdl > 1)
+      return CKV_ERR_INVALID_ARG;
+  }
   if (p->shared_elastic != 0 && p->shared_elastic != 1) return CKV_ERR_INVALID_ARG;
   if (p->global_alpha != 0 && p->global_alpha != 1) return CKV_ERR_INVALID_ARG;
   if (p->units_per_prompt < 0) return CKV_ERR_INVALID_ARG;
@@ -168,7 +204,8 @@ static cudaError_t launch_ws_reset(int* status, size_t n_flag_words, cudaStream_
 static ckv_status score_impl(const ckv_shape& s, const ckv_params& p, const void* q, const void* k,
                              const float* head_w, float* scores, float* colmass, char* ws, cudaStream_t st) {
   const WsLayout w = ws_layout(s, p);
-  const int path = g_score_path.load(std::memory_order_relaxed);
+  const CallTuning tune = t_call ? *t_call : resolve_tuning(p);
+  const int path = tune.score_path;
   const bool tc_ok = score_tc_supported(s) && s.seq_len >= 128;
   if (path == 2 && !tc_ok) return CKV_ERR_UNSUPPORTED;
   const bool use_tc = tc_ok && path != 1;
@@ -176,12 +213,12 @@ static ckv_status score_impl(const ckv_shape& s, const ckv_params& p, const void
   // status words keep a code that no ckv_device_status call has read yet
   CKV_CUDA(launch_ws_reset(reinterpret_cast<int*>(ws + w.status), use_tc ? tc_layout(s).flag_bytes / sizeof(int) : 0, st));
   float* csum = reinterpret_cast<float*>(ws + w.csum);
-  const cudaEvent_t ev0 = t_scan_start, ev1 = t_scan_stop;
+  const cudaEvent_t ev0 = tune.ev0, ev1 = tune.ev1;
   int* marker = reinterpret_cast<int*>(ws + w.status) + kPathMarkerWord;   // who wrote the row statistics
   if (use_tc) {
     // grouped output where it applies: both arrays fit the per-head region (at least two heads per group)
     TcGrouped grp{csum, csum + (int64_t)s.n_units * s.n_kv_heads * s.seq_len, head_w, p.head_w_stride_unit};
-    const bool grouped = score_tc_groupable(s, p) && g_group_fuse.load(std::memory_order_relaxed) != 0;
+    const bool grouped = score_tc_groupable(s, p) && tune.group_fuse != 0;
     if (ev0) CKV_CUDA(cudaEventRecord(ev0, st));
     CKV_CUDA(launch_score_tc(s, q, k, csum, grouped ? &grp : nullptr, ws + w.tc_part, ws + w.tc_stat,
                              reinterpret_cast<int*>(ws + w.tc_flags), reinterpret_cast<int*>(ws + w.status), st));
@@ -221,6 +258,7 @@ ckv_status ckv_score(const ckv_shape* shape, const ckv_params* params, const voi
                      const float* head_w, float* scores, float* colmass, void* ws, size_t ws_bytes, void* stream) {
   CKV_TRY(check_shape(shape));
   CKV_TRY(check_params(shape, params));
+  const TuningScope tuning_scope(*params);
   if (!all_aligned16({q_win, k}) || !all_aligned4({head_w, scores, colmass})) return CKV_ERR_INVALID_ARG;
   // the score stage alone uses the leading sections of the work space
   if (!ws || !aligned(ws, 256) || ws_bytes < ws_layout(*shape, *params).score_extent) return CKV_ERR_WORKSPACE;
@@ -232,6 +270,7 @@ ckv_status ckv_budget(const ckv_shape* shape, const ckv_params* params, const fl
                       void* ws, size_t ws_bytes, void* stream) {
   CKV_TRY(check_shape(shape));
   CKV_TRY(check_params(shape, params));
+  const TuningScope tuning_scope(*params);
   if (!all_aligned4({scores, colmass, sens, budgets, offsets, bucket, entropy})) return CKV_ERR_INVALID_ARG;
   CKV_TRY(check_ws(shape, params, ws, ws_bytes));
   const WsLayout w = ws_layout(*shape, *params);
@@ -246,6 +285,7 @@ ckv_status ckv_vnorm(const ckv_shape* shape, const ckv_params* params, const voi
                      float* scores_or_null, void* ws, size_t ws_bytes, void* stream) {
   CKV_TRY(check_shape(shape));
   CKV_TRY(check_params(shape, params));
+  const TuningScope tuning_scope(*params);
   if (!all_aligned16({v}) || !all_aligned4({rho})) return CKV_ERR_INVALID_ARG;
   if (scores_or_null && !aligned(scores_or_null, 4)) return CKV_ERR_INVALID_ARG;
   CKV_TRY(check_ws(shape, params, ws, ws_bytes));
@@ -261,6 +301,7 @@ ckv_status ckv_attend(const ckv_shape* shape, const ckv_params* params, const vo
                       float* out, float* lse, void* ws, size_t ws_bytes, void* stream) {
   CKV_TRY(check_shape(shape));
   CKV_TRY(check_params(shape, params));
+  const TuningScope tuning_scope(*params);
   if (n_dec < 1 || (shape->n_q_heads / shape->n_kv_heads) * n_dec > kAttendMaxRows) return CKV_ERR_UNSUPPORTED;
   if (compressed != 0 && compressed != 1) return CKV_ERR_INVALID_ARG;
   if (!all_aligned16({q_dec, k, v}) || !all_aligned4({out, lse})) return CKV_ERR_INVALID_ARG;
@@ -278,6 +319,7 @@ ckv_status ckv_kept_mass(const ckv_shape* shape, const ckv_params* params, const
                          size_t ws_bytes, void* stream) {
   CKV_TRY(check_shape(shape));
   CKV_TRY(check_params(shape, params));
+  const TuningScope tuning_scope(*params);
   if (!all_aligned16({q_win, k_out}) || !all_aligned4({indices, budgets, offsets, kept})) return CKV_ERR_INVALID_ARG;
   CKV_TRY(check_ws(shape, params, ws, ws_bytes));
   const WsLayout w = ws_layout(*shape, *params);
@@ -292,6 +334,7 @@ ckv_status ckv_prompt_mass(const ckv_shape* shape, const ckv_params* params, con
                            void* stream) {
   CKV_TRY(check_shape(shape));
   CKV_TRY(check_params(shape, params));
+  const TuningScope tuning_scope(*params);
   if (!params->global_alpha || !all_aligned4({colmass, pmass})) return CKV_ERR_INVALID_ARG;
   CKV_CUDA(launch_prompt_mass(*shape, *params, colmass, pmass, (cudaStream_t)stream));
   return CKV_OK;
@@ -301,6 +344,7 @@ ckv_status ckv_global_scores(const ckv_shape* shape, const ckv_params* params, c
                              const float* pmass, int32_t units_total, float* scores, float* colmass, void* stream) {
   CKV_TRY(check_shape(shape));
   CKV_TRY(check_params(shape, params));
+  const TuningScope tuning_scope(*params);
   if (!params->global_alpha || units_total < params->units_per_prompt) return CKV_ERR_INVALID_ARG;
   if (!all_aligned4({head_w, pmass, scores, colmass})) return CKV_ERR_INVALID_ARG;
   CKV_CUDA(launch_global_scores(*shape, *params, units_total, head_w, pmass, scores, colmass, (cudaStream_t)stream));
@@ -310,6 +354,7 @@ ckv_status ckv_global_scores(const ckv_shape* shape, const ckv_params* params, c
 ckv_status ckv_unit_max(const ckv_shape* shape, const ckv_params* params, float* scores, void* stream) {
   CKV_TRY(check_shape(shape));
   CKV_TRY(check_params(shape, params));
+  const TuningScope tuning_scope(*params);
   if (!all_aligned4({scores})) return CKV_ERR_INVALID_ARG;
   CKV_CUDA(launch_unit_max(*shape, scores, (cudaStream_t)stream));
   return CKV_OK;
@@ -319,6 +364,7 @@ ckv_status ckv_select(const ckv_shape* shape, const ckv_params* params, const fl
                       const int32_t* offsets, int32_t* indices, void* ws, size_t ws_bytes, void* stream) {
   CKV_TRY(check_shape(shape));
   CKV_TRY(check_params(shape, params));
+  const TuningScope tuning_scope(*params);
   if (!all_aligned4({scores, budgets, offsets, indices})) return CKV_ERR_INVALID_ARG;
   CKV_TRY(check_ws(shape, params, ws, ws_bytes));
   int* status = reinterpret_cast<int*>(static_cast<char*>(ws) + ws_layout(*shape, *params).status);
@@ -330,6 +376,7 @@ ckv_status ckv_gather(const ckv_shape* shape, const ckv_params* params, const vo
                       const int32_t* indices, const int32_t* offsets, void* k_out, void* v_out, void* stream) {
   CKV_TRY(check_shape(shape));
   CKV_TRY(check_params(shape, params));
+  const TuningScope tuning_scope(*params);
   if (!all_aligned16({k, v, k_out, v_out}) || !all_aligned4({indices, offsets})) return CKV_ERR_INVALID_ARG;
   CKV_CUDA(launch_gather(*shape, *params, k, v, indices, offsets, k_out, v_out, (cudaStream_t)stream));
   return CKV_OK;
@@ -341,6 +388,7 @@ ckv_status ckv_compress(const ckv_shape* shape, const ckv_params* params, const 
                         int32_t* bucket_or_null, float* entropy_or_null, void* ws, size_t ws_bytes, void* stream) {
   CKV_TRY(check_shape(shape));
   CKV_TRY(check_params(shape, params));
+  const TuningScope tuning_scope(*params);
   if (!all_aligned16({q_win, k, v, k_out, v_out}) || !all_aligned4({head_w, sens, indices, budgets, offsets}))
     return CKV_ERR_INVALID_ARG;
   if ((scores_or_null && !aligned(scores_or_null, 4)) || (bucket_or_null && !aligned(bucket_or_null, 4)) ||
@@ -438,6 +486,7 @@ ckv_status ckv_compress_host(const ckv_shape* shape, const ckv_params* params, c
                              void* ws, size_t ws_bytes, void* stream) {
   CKV_TRY(check_shape(shape));
   CKV_TRY(check_params(shape, params));
+  const TuningScope tuning_scope(*params);
   if (!q_win_host || !k_host || !v_host || !head_w_host || !sens_host || !k_out_host || !v_out_host ||
       !indices_host || !budgets_host || !offsets_host)
     return CKV_ERR_INVALID_ARG;
@@ -519,11 +568,13 @@ int ckv_set_tunable(const char* name, int value) {
   if (!name) return -1;
   if (std::string(name) == "group_fuse") return g_group_fuse.exchange(value != 0 ? 1 : 0);
   if (std::string(name) == "pdl") return g_pdl.exchange(value != 0 ? 1 : 0);
+  if (std::string(name) == "run_tiles") return value >= 1 && value <= 64 ? g_run_tiles.exchange(value) : -1;
+  if (std::string(name) == "l2_hints") return value == 0 || value == 1 ? g_l2_hints.exchange(value) : -1;
   if (std::string(name) == "wait_limit_us") {
     if (value < 1) return -1;
     return (int)(g_wait_limit_ns.exchange((unsigned long long)value * 1000ull) / 1000ull);
   }
-  return set_tc_tunable(name, value);
+  return -1;
 }
 
 int64_t ckv_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
@@ -602,6 +653,7 @@ extern "C" ckv_status ckv_score_noalloc(const ckv_shape* shape, const ckv_params
                                         void* stream) {
   CKV_TRY(check_shape(shape));
   CKV_TRY(check_params(shape, params));
+  const TuningScope tuning_scope(*params);
   if (!all_aligned16({q_win, k}) || !all_aligned4({head_w, scores, colmass})) return CKV_ERR_INVALID_ARG;
   if (ws_layout(*shape, *params).score_extent > (size_t)CKV_NOALLOC_SCRATCH_BYTES) return CKV_ERR_WORKSPACE;
   char* scratch = nullptr;

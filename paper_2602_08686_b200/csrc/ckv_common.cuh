@@ -61,7 +61,6 @@ struct TcLayout {
 };
 TcLayout tc_layout(const ckv_shape& s);
 bool score_tc_supported(const ckv_shape& s);
-int set_tc_tunable(const char* name, int value);
 // Grouped output of the scan (see score_tc.cu): per KV group the weighted maximum over its query heads and
 // their summed column mass, [Nu, Hkv, L] each, instead of the per-head column sums.  Possible when a group's
 // heads fill one row block, there are at least two of them and the pooling is max or none; requires
@@ -88,6 +87,9 @@ unsigned long long wait_limit_ns();
 // touches anything the predecessor wrote (or reads what it will overwrite); a predecessor lets it start early with
 // pdl_launch_dependents().  Both are no-ops in a kernel launched the ordinary way.
 bool pdl_enabled();
+// Scheduling settings of the call in progress on this thread (params->tuning over the process-wide defaults).
+int tuning_run_tiles();
+int tuning_l2_hints();
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 inline cudaLaunchAttribute pdl_attribute() {

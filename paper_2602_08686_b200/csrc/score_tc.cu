@@ -61,9 +61,6 @@ constexpr float kScale = 0.12751743074602467f;
 // UMMA instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = 128.
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 
-// Tunables of the schedule (process-wide; see ckv_set_tunable).
-std::atomic<int> g_run_tiles{16};       // key tiles per run
-std::atomic<int> g_l2_hints{1};         // 1: P1 loads keep their lines (evict_last), P2 loads release them
 
 struct TcArgs {
   int Nu, H, Hkv, G, L, W, n;
@@ -907,13 +904,6 @@ TcLayout tc_layout(const ckv_shape& s) {
   return t;
 }
 
-int set_tc_tunable(const char* name, int value) {
-  const std::string n(name);
-  if (n == "run_tiles" && value >= 1 && value <= 64) return g_run_tiles.exchange(value);
-  if (n == "l2_hints" && (value == 0 || value == 1)) return g_l2_hints.exchange(value);
-  return -1;
-}
-
 bool score_tc_groupable(const ckv_shape& s, const ckv_params& p) {
   const bool avg = p.pool_kind == CKV_POOL_AVG && p.pool_size / 2 > 0;
   return score_tc_supported(s) && tc_layout(s).RB == 1 && s.n_q_heads >= 2 * s.n_kv_heads && !avg;
@@ -930,7 +920,7 @@ cudaError_t launch_score_tc(const ckv_shape& s, const void* q, const void* k, fl
   a.Nu = s.n_units, a.H = s.n_q_heads, a.Hkv = s.n_kv_heads, a.G = a.H / a.Hkv, a.L = s.seq_len, a.W = s.window;
   a.n = a.L - a.W;
   a.RB = t.RB, a.hpb = kTile / a.W, a.T = t.T, a.C = (int)t.C;
-  a.run = g_run_tiles.load();
+  a.run = tuning_run_tiles();
   a.RPC = (a.T + a.run - 1) / a.run;
   if (t.C * a.RPC > (int64_t)1 << 30) return cudaErrorInvalidValue;
   a.NR = a.C * a.RPC;
@@ -941,7 +931,7 @@ cudaError_t launch_score_tc(const ckv_shape& s, const void* q, const void* k, fl
   const int t_last = a.T - (a.RPC - 1) * a.run;
   a.ppr = a.run < 2 ? 1 : 2;
   a.expected = (a.RPC - 1) * a.ppr + (t_last < 2 ? t_last : 2);
-  a.hints = g_l2_hints.load();
+  a.hints = tuning_l2_hints();
   const int hpb_box = a.hpb < a.H ? a.hpb : a.H;
   a.q_bytes = 2u * 64u * 2u * (uint32_t)a.W * (uint32_t)hpb_box;
   a.q_split = hpb_box * a.W < kTile;  // a short box would pack its halves closer than the operand layout wants

@@ -664,3 +664,59 @@ def test_two_streams_two_work_spaces(B):
             assert B.ckv_device_status(o["ws"]) == B.OK
             for key in ("scores", "indices", "budgets", "k_out", "v_out"):
                 assert torch.equal(o[key], serial[i][key]), (i, key)
+
+
+def test_per_call_tuning_on_two_threads(B):
+    """Scheduling settings travel with the call (params->tuning): two host threads, each on its own stream, run the
+    same problem with different settings (run length, L2 hints, dependent launches, score path; one of them with its
+    own event pair around the scan) at the same time.  Every call must give the default call's selection, and the
+    process-wide defaults must be what they were."""
+    import threading
+    cfg = gen.shrink(gen.CONFIGS["c2"], n_layers=3, seq_len=4200, budget_per_head=96, n_needles=4)
+    b = gen.make_batch(cfg, "cuda")
+    P = params_of(B, problem_of(cfg, 3))
+    want = B.compress(b["q"], b["k"], b["v"], b["head_w"], b["sens"], P, want_scores=True)
+    plain = B.compress(b["q"], b["k"], b["v"], b["head_w"], b["sens"], P, want_scores=True,
+                       tuning=B.make_tuning(score_path=1))
+    torch.cuda.synchronize()
+    ev = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+    ev[0].record(), ev[1].record()
+    torch.cuda.synchronize()
+    tunings = [B.make_tuning(run_tiles=3, l2_hints=0, pdl=0, score_path=2, scan_events=ev),
+               B.make_tuning(run_tiles=40, group_fuse=1, pdl=1), B.make_tuning(score_path=1)]
+    results, errors = [[] for _ in tunings], []
+
+    def worker(i):
+        try:
+            st = torch.cuda.Stream()
+            with torch.cuda.stream(st):
+                for _ in range(5):
+                    results[i].append(B.compress(b["q"], b["k"], b["v"], b["head_w"], b["sens"], P, want_scores=True,
+                                                 stream=st, tuning=tunings[i]))
+            st.synchronize()
+        except Exception as e:      # noqa: BLE001 -- reported by the main thread
+            errors.append(e)
+
+    threads = [threading.Thread(target=worker, args=(i,)) for i in range(len(tunings))]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    torch.cuda.synchronize()
+    for i, outs_i in enumerate(results):
+        ref = plain if i == 2 else want       # the plain kernels round differently from the tensor-core scan
+        for o in outs_i:
+            assert B.ckv_device_status(o["ws"]) == B.OK
+            if i < 2:     # other run length: the row statistics are merged in another order, the last bits may differ
+                rel = ((o["scores"] - ref["scores"]).abs() / ref["scores"].abs().clamp_min(1e-20)).max().item()
+                assert rel < 1e-5, rel
+                assert torch.equal(o["scores"], outs_i[0]["scores"])      # and every call with one setting agrees
+            else:
+                assert torch.equal(o["scores"], ref["scores"]) and torch.equal(o["indices"], ref["indices"])
+    assert ev[0].elapsed_time(ev[1]) > 0.0           # the first thread's scan was bracketed by its own events
+    again = B.compress(b["q"], b["k"], b["v"], b["head_w"], b["sens"], P, want_scores=True)
+    assert torch.equal(again["scores"], want["scores"]) and torch.equal(again["indices"], want["indices"])
+    # out-of-range settings are argument errors
+    with pytest.raises(B.CkvError):
+        B.compress(b["q"], b["k"], b["v"], b["head_w"], b["sens"], P, tuning=B.make_tuning(run_tiles=65))

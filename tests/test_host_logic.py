@@ -97,6 +97,16 @@ def test_argument_errors_are_found_on_the_host():
     one = llama_shape(Nu=1)
     one.q_stride_unit = one.kv_stride_unit = 0
     assert B.ckv_workspace_bytes(one, p) > 0
+    # per-call scheduling settings: -1 or a value in range
+    for field, value in (("run_tiles", 0), ("run_tiles", 65), ("score_path", 3), ("l2_hints", 2), ("pdl", -2)):
+        t = B.make_tuning()
+        setattr(t, field, value)
+        bad_t = default_params()
+        bad_t.tuning = C.pointer(t)
+        assert score(s, bad_t) == B.ERR_INVALID_ARG, field
+    ok_t = default_params()
+    ok_t.tuning = C.pointer(B.make_tuning(run_tiles=8, pdl=0))
+    assert B.ckv_workspace_bytes(s, ok_t) == B.ckv_workspace_bytes(s, p)
     # the four-axis gate table: its sizes must be given, and it is one table for all units
     coords = C.cast(fake, C.c_void_p)
     gate = default_params(n_buckets=20)
