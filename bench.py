@@ -43,9 +43,9 @@ FALLBACK_HBM_GBS = 6650.0
 # describe the kernel that is timed and the line says null.
 SCAN_SOURCE = os.path.join(ROOT, "paper_2602_08686_b200", "csrc", "score_tc.cu")
 SCAN_DRAM_TRAFFIC_PER_UNIT = {
-    "c2": {"source": "a7657adb4bc3", "bytes": (1.019321e9 + 8.769792e6) / 8},
-    "c3": {"source": "a7657adb4bc3", "bytes": (1.019321e9 + 8.769792e6) / 8},
-    "c4": {"source": "a7657adb4bc3", "bytes": (1.015547392e9 + 7.609344e6) / 2},
+    "c2": {"source": "4ebc2264eec8", "bytes": (1.019676e9 + 8.599552e6) / 8},
+    "c3": {"source": "4ebc2264eec8", "bytes": (1.019676e9 + 8.599552e6) / 8},
+    "c4": {"source": "4ebc2264eec8", "bytes": (1.014877952e9 + 7.403008e6) / 2},
 }
 
 
