@@ -34,6 +34,11 @@ def draw(seed):
     layers = int(r.integers(1, 4)) * 2
     modes = dict(value_norm=bool(r.integers(0, 2)), shared_elastic=bool(r.integers(0, 4) == 0),
                  global_alpha=bool(r.integers(0, 4) == 0), units_per_prompt=2)
+    # a third of the cases take their threshold from the four-axis gate table; every case carries its own scheduling
+    # settings (they must not change any result)
+    modes["gate"] = (int(r.integers(1, 5)), int(r.integers(1, 5)), int(r.integers(1, 4))) if r.integers(0, 3) == 0 else None
+    modes["tuning"] = dict(run_tiles=int(r.integers(1, 41)), l2_hints=int(r.integers(0, 2)), pdl=int(r.integers(0, 2)),
+                           group_fuse=int(r.integers(0, 2)))
     cfg = gen.shrink(gen.CONFIGS["c2"], config_id=100 + seed, n_layers=layers, batch=1, n_q_heads=Hkv * G, n_kv_heads=Hkv,
                      seq_len=L, window=W, pool_kind=pool_kind, pool_size=pool_size, budget_per_head=budget,
                      floor_per_head=floor, n_needles=2 if n > 64 else 0, dtype=dtype, n_buckets=int(r.choice([1, 7, 16])))
@@ -43,18 +48,33 @@ def draw(seed):
 @pytest.mark.parametrize("seed", range(100))
 def test_random_case(B, seed):
     cfg, modes = draw(seed)
+    gate, tuning = modes.pop("gate", None), modes.pop("tuning", None)
     Nu = cfg.n_units
     b = gen.make_batch(cfg, "cpu")
     # thresholds near the bulk of the scores, so that the candidate counts differ between heads
     prob = problem_of(cfg, Nu, **modes)
     qn, kn, vn, hw = (gen.as_numpy(b[x]) for x in ("q", "k", "v", "head_w"))
     sc, cm = oracle.score(prob, qn, kn, hw, v=vn if modes["value_norm"] else None)
-    qs = np.quantile(sc, np.linspace(0.3, 0.995, cfg.n_buckets)).astype(np.float32)
-    sens = torch.from_numpy(qs[np.random.default_rng(seed).permutation(cfg.n_buckets)].copy())
+    rs = np.random.default_rng(seed)
+    coords, gate_kw = None, {}
+    if gate is None:
+        qs = np.quantile(sc, np.linspace(0.3, 0.995, cfg.n_buckets)).astype(np.float32)
+        sens = torch.from_numpy(qs[rs.permutation(cfg.n_buckets)].copy())
+    else:       # T_gate[layer, entropy bin, perplexity bin, budget level], thresholds from the same quantile range
+        n_l, n_p, n_b = gate
+        cells = n_l * cfg.n_buckets * n_p * n_b
+        qs = np.quantile(sc, np.linspace(0.3, 0.995, cells)).astype(np.float32)
+        sens = torch.from_numpy(qs[rs.permutation(cells)].reshape(n_l, cfg.n_buckets, n_p, n_b).copy())
+        coords = np.stack([rs.integers(0, n_l, Nu), rs.integers(0, n_p, Nu), rs.integers(0, n_b, Nu)], 1).astype(np.int32)
+        gate_kw = dict(gate_layers=n_l, ppl_bins=n_p, budget_levels=n_b)
     P = params_of(B, prob)
     for f in ("value_norm", "shared_elastic", "global_alpha", "units_per_prompt"):
         setattr(P, f, modes[f])
-    out = B.compress(*(b[x].cuda() for x in ("q", "k", "v", "head_w")), sens.cuda(), P, want_scores=True)
+    if gate is not None:
+        P.n_gate_layers, P.n_ppl_bins, P.n_budget_levels = gate
+    out = B.compress(*(b[x].cuda() for x in ("q", "k", "v", "head_w")), sens.cuda(), P, want_scores=True,
+                     gate_coords=None if coords is None else torch.from_numpy(coords).cuda(),
+                     tuning=None if tuning is None else B.make_tuning(**tuning))
     assert B.ckv_device_status(out["ws"]) == B.OK
     gs = out["scores"].double().cpu().numpy()
     rel = np.abs(gs - sc) / np.maximum(np.abs(sc), 1e-20)
@@ -62,7 +82,8 @@ def test_random_case(B, seed):
     idx, bud, off = (out[x].cpu().numpy() for x in ("indices", "budgets", "offsets"))
     bucket = out["bucket"].cpu().numpy()
     for u in range(Nu):
-        prob_u = problem_of(cfg, 1, bucket_override=int(bucket[u]), shared_elastic=modes["shared_elastic"])
+        prob_u = problem_of(cfg, 1, bucket_override=int(bucket[u]), shared_elastic=modes["shared_elastic"],
+                            gate_coords=None if coords is None else coords[u:u + 1], **gate_kw)
         mine = oracle.budget(prob_u, gs[u:u + 1], cm[u:u + 1], sens.numpy())
         assert (mine["budgets"][0] == bud[u]).all(), (u, mine["budgets"], bud[u], cfg, modes)
     want = oracle.select(prob, gs, bud, off)
@@ -82,7 +103,8 @@ def draw_long(seed):
                      pool_size=int(r.choice([3, 7])), budget_per_head=int(r.integers(W + 64, 3000)),
                      floor_per_head=int(r.integers(0, 9)), n_needles=8)
     modes = dict(value_norm=bool(r.integers(0, 2)), shared_elastic=False, global_alpha=bool(r.integers(0, 3) == 0),
-                 units_per_prompt=2)
+                 units_per_prompt=2, gate=(2, 4, 2) if seed % 3 == 0 else None,
+                 tuning=dict(run_tiles=int(r.integers(2, 33)), pdl=int(r.integers(0, 2))))
     return cfg, modes
 
 
