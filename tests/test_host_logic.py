@@ -37,6 +37,36 @@ def test_library_exports_every_declared_symbol():
     assert B.status_string(B.ERR_TIMEOUT)
 
 
+def test_header_is_plain_c_and_links(tmp_path):
+    """The boundary is a C ABI: the header compiles as C99 and a C program that only knows the header links
+    against the library and gets the host-side answers (no GPU involved)."""
+    src = tmp_path / "abi.c"
+    src.write_text(r"""
+#include <stdio.h>
+#include <string.h>
+#include "ckv.h"
+int main(void) {
+  ckv_shape s; ckv_params p;
+  memset(&s, 0, sizeof s); memset(&p, 0, sizeof p);
+  s.n_units = 2; s.n_q_heads = 32; s.n_kv_heads = 8; s.head_dim = 128; s.seq_len = 4096; s.window = 32; s.dtype = CKV_BF16;
+  s.q_stride_row = 128; s.q_stride_head = 32 * 128; s.q_stride_unit = 32 * 32 * 128;
+  s.kv_stride_tok = 128; s.kv_stride_head = 4096 * 128; s.kv_stride_unit = 8 * 4096 * 128;
+  p.pool_kind = CKV_POOL_MAX; p.pool_size = 7; p.budget_per_head = 512; p.floor_per_head = 1; p.n_buckets = 16;
+  p.bucket_override = -1; p.head_w_stride_unit = 32;
+  printf("%d %zu %zu %s\n", ckv_version(), ckv_workspace_bytes(&s, &p), ckv_score_workspace_bytes(&s, &p),
+         ckv_status_string(CKV_ERR_TIMEOUT));
+  s.head_dim = 64;
+  return ckv_workspace_bytes(&s, &p) == 0 ? 0 : 1;
+}
+""")
+    exe = tmp_path / "abi"
+    libdir = os.path.dirname(B.LIB_PATH)
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Werror", "-pedantic", "-I", os.path.join(ROOT, "include"), str(src),
+                           "-o", str(exe), "-L", libdir, "-l:libckv.so", "-Wl,-rpath," + libdir])
+    out = subprocess.run([str(exe)], stdout=subprocess.PIPE, check=True).stdout.decode().split()
+    assert int(out[0]) >= 100 and int(out[1]) > int(out[2]) > 0
+
+
 def llama_shape(L=32768, W=32, Nu=2, H=32, Hkv=8, d=128, dtype=B.BF16):
     return B.ckv_shape(Nu, H, Hkv, d, L, W, dtype, 0, H * W * d, W * d, d, Hkv * L * d, L * d, d)
 
