@@ -318,7 +318,8 @@ ckv_status ckv_device_status(const void* ws, void* stream);
 
 /* Diagnostic switch for the window-score scan: 0 = automatic (tensor-core kernel for bf16 inputs with
  * window 16, 32 or 64 and L >= 128, plain kernels otherwise), 1 = always the plain kernels, 2 = require
- * the tensor-core kernel (ckv_score returns CKV_ERR_UNSUPPORTED where it does not apply).  Process-wide;
+ * the tensor-core kernel (ckv_score returns CKV_ERR_UNSUPPORTED where it does not apply).  Process-wide default
+ * (a call may carry its own in params->tuning);
  * returns the previous setting, or -1 for an invalid value. */
 int ckv_set_score_path(int path);
 
@@ -329,7 +330,7 @@ int ckv_set_score_path(int path);
  * thread: calls made from other threads are not affected and record nothing. */
 void ckv_set_scan_events(void* start_event, void* stop_event);
 
-/* Diagnostic knobs of the tensor-core scan (process-wide; the scores do not depend on them):
+/* Diagnostic knobs of the tensor-core scan (process-wide defaults, see ckv_tuning; the scores do not depend on them):
  *   "run_tiles"      key tiles per run, the unit CTAs take work in (1..64, default 16);
  *   "l2_hints"       1 (default): first-pass K loads ask L2 to keep their lines and second-pass loads
  *                    release them; 0: no hints;
