@@ -37,7 +37,7 @@ METRIC = "prefill_tokens_compressed_per_sec_per_layer"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of score_tc_kernel per unit, from ncu captures of small launches of
-# the workload's shape (profiles/score_tc_kernel_c2_8units.md: 8 units; 2 units for the 128k shape).  A launch's
+# the workload's shape (profiles/score_tc_kernel_c2_8units.md: 8 units; 2 units for the 128k shape; all 112 of config 5).  A launch's
 # traffic is this times its units (every unit streams its own K once per pass).  Each entry names the kernel source
 # it was taken from (first 12 hex digits of its SHA-256): when the source has changed since, the counters no longer
 # describe the kernel that is timed and the line says null.
@@ -46,6 +46,7 @@ SCAN_DRAM_TRAFFIC_PER_UNIT = {
     "c2": {"source": "4ebc2264eec8", "bytes": (1.019676e9 + 8.599552e6) / 8},
     "c3": {"source": "4ebc2264eec8", "bytes": (1.019676e9 + 8.599552e6) / 8},
     "c4": {"source": "4ebc2264eec8", "bytes": (1.014877952e9 + 7.403008e6) / 2},
+    "c5": {"source": "4ebc2264eec8", "bytes": (1.821095936e9 + 5.0745088e7) / 112},   # the whole workload was captured
 }
 
 
